@@ -1,0 +1,155 @@
+/* ptqtp.h -- C ABI of the PTQTP dual-trit-plane decode linear layer for NVIDIA B200 (sm_100a).
+ *
+ * A weight matrix W [N out, K in] is stored as two ternary planes T1, T2 in {-1,0,+1}^{N x K} and
+ * two scale tables alpha1, alpha2 with one fp16 value per output row per group of 128 input columns
+ * (Eq. 1-2: W ~ diag(alpha1) T1 + diag(alpha2) T2; Sec. 2.3 "Batch Processing": the scales are
+ * per group-row after reshaping n x d to (nd/G) x G with G = 128).  The layer computes
+ *
+ *     y[i] = sum_g ( alpha1[i,g] * sum_{j in g} T1[i,j] x[j]  +  alpha2[i,g] * sum_{j in g} T2[i,j] x[j] )
+ *
+ * where a trit contributes +x, -x or nothing (Sec. 4 "Hardware Efficiency") and the per-group
+ * scale is the only multiplication.
+ *
+ * Conventions for every call
+ *   - Pointers marked "device" are CUDA device pointers on the current device; "host" are host
+ *     pointers.  The caller owns every buffer.  Except where an entry point says otherwise the
+ *     library never allocates, frees or synchronises: calls enqueue work on `stream` (a
+ *     cudaStream_t passed as void*, NULL = the default stream) and return after the launch.
+ *   - Device buffers must be 16-byte aligned (PTQTP_ERR_ALIGN otherwise).
+ *   - Host-detectable errors return a negative status and launch nothing.
+ *   - Errors only the device can see (a plane entry outside {-1,0,1}, a bad header) are written
+ *     to `*dev_status` (a device int32 the caller zeroes beforehand and reads after syncing); the
+ *     kernel still completes normally.  `dev_status` may be NULL where noted.
+ *   - K must be a positive multiple of 128 (the group reshape of Sec. 2.3 presumes it); N >= 1.
+ *   - Matrices are row-major: T[i*K + j], alpha[i*(K/128) + g], X[m*K + j], Y[m*N + i].
+ *   - fp16 values cross the ABI as their 16-bit patterns (uint16_t).
+ *
+ * Packed format "PTQTP-B200 v1" (chosen for 128-bit coalesced streaming; the storage model of
+ * Appendix B "Memory Saving": 2 bits per trit per plane + one fp16 scale per plane per group):
+ *   [0, 256)            header: magic "PTQTPB2\0", u32 version(1), u32 format(1), i32 N, i32 K,
+ *                       i32 group(128), i32 K_pad, u64 codes_offset, u64 scales_offset, u64 total bytes
+ *   codes  (at 256)     N * (K_pad/1024) chunks of 512 bytes, row-major in (row, slice).  K_pad = K
+ *                       rounded up to a multiple of 1024; padding columns hold trit 0.
+ *                       Chunk (i, s) covers columns s*1024 .. s*1024+1023 of row i as 32 lane blocks
+ *                       of 16 bytes; lane block l covers the 32 columns s*1024 + 32*l + e, e = 0..31,
+ *                       as four little-endian u32 words:
+ *                         word 0: plane 1, e = 0..15      word 1: plane 1, e = 16..31
+ *                         word 2: plane 2, e = 0..15      word 3: plane 2, e = 16..31
+ *                       In a word, column offset e' = e mod 16 sits in the 16-bit half h = e'/8 at bits
+ *                       [16h + 2(e' mod 8), +1] as the code q = trit + 1 in {0,1,2} (3 never occurs).
+ *   scales (after codes) N * (K_pad/128) pairs (alpha1 fp16, alpha2 fp16), row-major; pairs of
+ *                       padding groups are zero.
+ *   ptqtp_packed_size = 256 + N*K_pad/2 + 4*N*K_pad/128 bytes, i.e. the Appendix B figure
+ *   2*N*K*2 + (K/128)*2*N*16 bits plus the header and the K padding.
+ */
+#ifndef PTQTP_H
+#define PTQTP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define PTQTP_API __attribute__((visibility("default")))
+#else
+#define PTQTP_API
+#endif
+
+typedef enum {
+    PTQTP_OK = 0,
+    PTQTP_ERR_NULL = -1,    /* a required pointer is NULL                                   */
+    PTQTP_ERR_SHAPE = -2,   /* N <= 0, K <= 0, K % 128 != 0, group != 128, M out of range   */
+    PTQTP_ERR_ALIGN = -3,   /* a device pointer is not 16-byte aligned                      */
+    PTQTP_ERR_SIZE = -4,    /* packed buffer smaller than ptqtp_packed_size                 */
+    PTQTP_ERR_TRIT = -5,    /* a plane entry outside {-1,0,1} (reported through dev_status) */
+    PTQTP_ERR_FORMAT = -6,  /* bad magic / version / shape in a packed header               */
+    PTQTP_ERR_CUDA = -7,    /* a CUDA runtime call failed; see ptqtp_last_cuda_error        */
+    PTQTP_ERR_CONFIG = -8   /* an expert launch configuration is not supported              */
+} ptqtp_status;
+
+typedef struct {
+    int32_t n_out;   /* N: output features (rows of W)            */
+    int32_t k_in;    /* K: input features, multiple of 128        */
+    int32_t group;   /* scale group size along K; must be 128     */
+    int32_t format;  /* packed format id; must be 1               */
+} ptqtp_shape;
+
+#define PTQTP_GROUP 128
+#define PTQTP_FORMAT_V1 1
+#define PTQTP_HEADER_BYTES 256
+#define PTQTP_MAX_BATCH 64
+
+/* Size in bytes of the packed blob for `shape` (header and padding included); 0 on a bad shape.
+ * Storage model: Appendix B "Memory Saving" (2 bits per trit, fp16 scales per group). */
+PTQTP_API size_t ptqtp_packed_size(const ptqtp_shape *shape /* host */);
+
+/* Pack planes and scales into the streaming format (hot-path step "pack"; one-time per matrix).
+ * T1, T2: device int8 [N*K], entries must be in {-1,0,1}; alpha1, alpha2: device fp16 bits [N*K/128];
+ * packed: device, at least ptqtp_packed_size bytes, fully overwritten; dev_status: device int32 or
+ * NULL -- receives PTQTP_ERR_TRIT if an entry is out of range (that entry is stored as 0).
+ * Defines the representation of Eq. 1-2 / Appendix B used by every other call. */
+PTQTP_API ptqtp_status ptqtp_pack(const ptqtp_shape *shape /* host */, const int8_t *T1, const int8_t *T2,
+                        const uint16_t *alpha1, const uint16_t *alpha2, void *packed,
+                        size_t packed_bytes, int32_t *dev_status, void *stream);
+
+/* Exact inverse of ptqtp_pack: recovers the int8 planes and the fp16 scale bit patterns.
+ * dev_status (device int32 or NULL) receives PTQTP_ERR_FORMAT if the blob's header does not match
+ * `shape`; outputs are then unspecified. */
+PTQTP_API ptqtp_status ptqtp_unpack(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
+                          int8_t *T1, int8_t *T2, uint16_t *alpha1, uint16_t *alpha2,
+                          int32_t *dev_status, void *stream);
+
+/* Batch-1 decode layer y = alpha1 (.) (T1 x) + alpha2 (.) (T2 x) (Eq. 1-2 with Sec. 2.3 groups;
+ * Sec. 4: additions/subtractions of x, one scale multiply per group and plane).
+ * packed: device blob from ptqtp_pack (its header is not re-read; `shape` is trusted);
+ * x: device fp16 [K]; y: device fp16 [N], fully overwritten.  x and y must not alias packed.
+ * Arithmetic: fp16 x, short fp16 partial sums flushed into fp32 accumulators, fp32 scale
+ * epilogue, one rounding to fp16 at the store.  Non-finite x gives unspecified non-finite y. */
+PTQTP_API ptqtp_status ptqtp_gemv(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
+                        const uint16_t *x, uint16_t *y, void *stream);
+
+/* Small-batch variant: Y[m,:] = layer(X[m,:]) for m < M, 1 <= M <= PTQTP_MAX_BATCH.
+ * X: device fp16 [M*K] row-major; Y: device fp16 [M*N] row-major.  Same definition per row of X. */
+PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, const void *packed,
+                               size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
+                               void *stream);
+
+/* End-to-end convenience for callers holding activations on the host: copies x_host [K] (host,
+ * ideally pinned) to x_dev, runs ptqtp_gemv, copies y_dev to y_host [N]; all three enqueued on
+ * `stream`, no synchronisation.  x_dev [K] and y_dev [N] are caller-owned device staging buffers. */
+PTQTP_API ptqtp_status ptqtp_gemv_host(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
+                             const uint16_t *x_host, uint16_t *y_host, uint16_t *x_dev, uint16_t *y_dev,
+                             void *stream);
+
+/* Expert entry point: ptqtp_gemv with an explicit launch configuration, for tuning and tests.
+ * rows_per_warp in {1,2,4}; k_split (warps of a CTA sharing a row, splitting K; must divide
+ * K_pad/1024) in {1,2,4,8}; ctas_per_sm >= 1 bounds the persistent grid (grid = min(tiles,
+ * ctas_per_sm * SM count)); depth = 128-bit loads per row kept in flight per lane (1,2,4,8; not
+ * every combination with rows_per_warp is built); 0 in any of these selects the library's own choice.
+ * arith: accumulation of the sign-selected activations -- 0 = fp32 accumulator fed by mixed-precision
+ * FMAs (fp16 operands), 1 = fp16x2 chains of 4 flushed into fp32, 2 = chains of 8, -1 = library choice.
+ * PTQTP_ERR_CONFIG if the combination is not built. */
+PTQTP_API ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
+                            const uint16_t *x, uint16_t *y, int32_t rows_per_warp, int32_t k_split,
+                            int32_t ctas_per_sm, int32_t depth, int32_t arith, void *stream);
+
+/* Parse the 256-byte header of a packed blob that was copied to the host (e.g. read from a file).
+ * Fills *shape and returns PTQTP_OK, or PTQTP_ERR_FORMAT / PTQTP_ERR_SIZE / PTQTP_ERR_NULL. */
+PTQTP_API ptqtp_status ptqtp_parse_header(const void *header_host, size_t bytes, ptqtp_shape *shape /* host */);
+
+/* Human-readable name of a status code (static storage, never NULL). */
+PTQTP_API const char *ptqtp_status_string(ptqtp_status status);
+
+/* The cudaError_t (as int) behind the calling thread's most recent PTQTP_ERR_CUDA, else 0. */
+PTQTP_API int ptqtp_last_cuda_error(void);
+
+/* Library version: major*10000 + minor*100 + patch. */
+PTQTP_API int ptqtp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PTQTP_H */

@@ -1,0 +1,199 @@
+"""ctypes binding of libptqtp.so: argument marshalling only; every step runs in the CUDA kernels.
+
+torch supplies device memory and streams.  Function names mirror the C ABI (include/ptqtp.h).
+There is no CPU path: if the shared library is missing or a call fails, a PtqtpError is raised.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libptqtp.so")
+
+GROUP = 128
+FORMAT_V1 = 1
+HEADER_BYTES = 256
+MAX_BATCH = 64
+
+OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_SIZE, ERR_TRIT, ERR_FORMAT, ERR_CUDA, ERR_CONFIG = (
+    0, -1, -2, -3, -4, -5, -6, -7, -8)
+
+EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny",
+           "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
+           "ptqtp_last_cuda_error", "ptqtp_version")
+
+
+class PtqtpError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        super().__init__("%s failed: %s (status %d, cuda error %d)"
+                         % (what, status_string(status), status, lib().ptqtp_last_cuda_error()))
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("n_out", ctypes.c_int32), ("k_in", ctypes.c_int32), ("group", ctypes.c_int32),
+                ("format", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libptqtp.so (built in-tree by build.py).  Raises if it is absent: no fallback exists."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libptqtp.so not found at %s: run `python -m paper_2509_16989_b200.build`"
+                               % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, i32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32
+        sp = ctypes.POINTER(Shape)
+        L.ptqtp_packed_size.restype = sz
+        L.ptqtp_packed_size.argtypes = [sp]
+        L.ptqtp_pack.restype = ctypes.c_int
+        L.ptqtp_pack.argtypes = [sp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.ptqtp_unpack.restype = ctypes.c_int
+        L.ptqtp_unpack.argtypes = [sp, vp, sz, vp, vp, vp, vp, vp, vp]
+        L.ptqtp_gemv.restype = ctypes.c_int
+        L.ptqtp_gemv.argtypes = [sp, vp, sz, vp, vp, vp]
+        L.ptqtp_gemm_skinny.restype = ctypes.c_int
+        L.ptqtp_gemm_skinny.argtypes = [sp, vp, sz, i32, vp, vp, vp]
+        L.ptqtp_gemv_host.restype = ctypes.c_int
+        L.ptqtp_gemv_host.argtypes = [sp, vp, sz, vp, vp, vp, vp, vp]
+        L.ptqtp_gemv_cfg.restype = ctypes.c_int
+        L.ptqtp_gemv_cfg.argtypes = [sp, vp, sz, vp, vp, i32, i32, i32, i32, i32, vp]
+        L.ptqtp_parse_header.restype = ctypes.c_int
+        L.ptqtp_parse_header.argtypes = [vp, sz, sp]
+        L.ptqtp_status_string.restype = ctypes.c_char_p
+        L.ptqtp_status_string.argtypes = [ctypes.c_int]
+        L.ptqtp_last_cuda_error.restype = ctypes.c_int
+        L.ptqtp_version.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status):
+    return lib().ptqtp_status_string(int(status)).decode()
+
+
+def make_shape(N, K, group=GROUP, fmt=FORMAT_V1):
+    return Shape(int(N), int(K), int(group), int(fmt))
+
+
+def packed_size(N, K):
+    return int(lib().ptqtp_packed_size(ctypes.byref(make_shape(N, K))))
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dev(t, dtype, what):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError("%s must be a contiguous CUDA tensor of dtype %s" % (what, dtype))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _check(status, what):
+    if status != OK:
+        raise PtqtpError(status, what)
+
+
+def ptqtp_pack(T1, T2, alpha1, alpha2, packed=None, dev_status=None, stream=None):
+    """Pack int8 planes [N,K] and fp16 scales [N,K/128] (CUDA tensors).  Returns (packed uint8 tensor, dev_status)."""
+    N, K = T1.shape
+    shape = make_shape(N, K)
+    nbytes = packed_size(N, K)
+    if nbytes == 0:
+        raise PtqtpError(ERR_SHAPE, "ptqtp_packed_size")
+    if packed is None:
+        packed = torch.empty(nbytes, dtype=torch.uint8, device=T1.device)
+    if dev_status is None:
+        dev_status = torch.zeros(1, dtype=torch.int32, device=T1.device)
+    st = lib().ptqtp_pack(ctypes.byref(shape), _dev(T1, torch.int8, "T1"), _dev(T2, torch.int8, "T2"),
+                          _dev(alpha1, torch.float16, "alpha1"), _dev(alpha2, torch.float16, "alpha2"),
+                          _dev(packed, torch.uint8, "packed"), packed.numel(),
+                          _dev(dev_status, torch.int32, "dev_status"), _stream_ptr(stream))
+    _check(st, "ptqtp_pack")
+    return packed, dev_status
+
+
+def ptqtp_unpack(packed, N, K, dev_status=None, stream=None):
+    """Inverse of ptqtp_pack.  Returns (T1, T2, alpha1, alpha2, dev_status) as CUDA tensors."""
+    shape = make_shape(N, K)
+    dev = packed.device
+    T1 = torch.empty((N, K), dtype=torch.int8, device=dev)
+    T2 = torch.empty((N, K), dtype=torch.int8, device=dev)
+    a1 = torch.empty((N, K // GROUP), dtype=torch.float16, device=dev)
+    a2 = torch.empty((N, K // GROUP), dtype=torch.float16, device=dev)
+    if dev_status is None:
+        dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = lib().ptqtp_unpack(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
+                            _dev(T1, torch.int8, "T1"), _dev(T2, torch.int8, "T2"),
+                            _dev(a1, torch.float16, "alpha1"), _dev(a2, torch.float16, "alpha2"),
+                            _dev(dev_status, torch.int32, "dev_status"), _stream_ptr(stream))
+    _check(st, "ptqtp_unpack")
+    return T1, T2, a1, a2, dev_status
+
+
+def ptqtp_gemv(packed, N, K, x, y=None, stream=None):
+    """y[N] = layer(x[K]) from a packed blob; fp16 CUDA tensors."""
+    shape = make_shape(N, K)
+    if y is None:
+        y = torch.empty(N, dtype=torch.float16, device=x.device)
+    st = lib().ptqtp_gemv(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
+                          _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"), _stream_ptr(stream))
+    _check(st, "ptqtp_gemv")
+    return y
+
+
+def ptqtp_gemv_cfg(packed, N, K, x, y=None, rows_per_warp=0, k_split=0, ctas_per_sm=0, depth=0, arith=-1,
+                   stream=None):
+    shape = make_shape(N, K)
+    if y is None:
+        y = torch.empty(N, dtype=torch.float16, device=x.device)
+    st = lib().ptqtp_gemv_cfg(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
+                              _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"),
+                              int(rows_per_warp), int(k_split), int(ctas_per_sm), int(depth), int(arith),
+                              _stream_ptr(stream))
+    _check(st, "ptqtp_gemv_cfg")
+    return y
+
+
+def ptqtp_gemm_skinny(packed, N, K, X, Y=None, stream=None):
+    """Y[M,N] = layer applied to each row of X[M,K]; fp16 CUDA tensors, 1 <= M <= 64."""
+    shape = make_shape(N, K)
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=X.device)
+    st = lib().ptqtp_gemm_skinny(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
+                                 int(M), _dev(X, torch.float16, "X"), _dev(Y, torch.float16, "Y"),
+                                 _stream_ptr(stream))
+    _check(st, "ptqtp_gemm_skinny")
+    return Y
+
+
+def ptqtp_gemv_host(packed, N, K, x_host, y_host, x_dev, y_dev, stream=None):
+    """Host-buffer call: H2D copy of x, GEMV, D2H copy of y, all on `stream` (no sync)."""
+    shape = make_shape(N, K)
+    for t, what in ((x_host, "x_host"), (y_host, "y_host")):
+        if t.is_cuda or t.dtype != torch.float16 or not t.is_contiguous():
+            raise TypeError("%s must be a contiguous fp16 host tensor" % what)
+    st = lib().ptqtp_gemv_host(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
+                               ctypes.c_void_p(x_host.data_ptr()), ctypes.c_void_p(y_host.data_ptr()),
+                               _dev(x_dev, torch.float16, "x_dev"), _dev(y_dev, torch.float16, "y_dev"),
+                               _stream_ptr(stream))
+    _check(st, "ptqtp_gemv_host")
+    return y_host
+
+
+def ptqtp_parse_header(header_bytes):
+    """Parse a host copy (bytes) of a blob's header; returns (N, K)."""
+    buf = ctypes.create_string_buffer(bytes(header_bytes), len(header_bytes))
+    shape = Shape()
+    st = lib().ptqtp_parse_header(ctypes.cast(buf, ctypes.c_void_p), len(header_bytes), ctypes.byref(shape))
+    _check(st, "ptqtp_parse_header")
+    return shape.n_out, shape.k_in

@@ -1,0 +1,124 @@
+"""CPU-only checks of the C ABI: the library builds, loads and exports what include/ptqtp.h declares,
+host-side validation returns the documented codes, and the size/header helpers agree with the
+independent format description.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import packed_format as pf
+from paper_2509_16989_b200 import binding, build
+from paper_2509_16989_b200.inputs import make_case
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    build.build()
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "ptqtp.h")).read()
+    return sorted(set(re.findall(r"PTQTP_API[^;(]*?\b(ptqtp_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = declared_symbols()
+    assert len(names) >= 11 and set(names) == set(binding.EXPORTS)
+    for n in names:
+        assert getattr(L, n) is not None
+    assert L.ptqtp_version() >= 100
+
+
+def test_packed_size_is_memory_formula_plus_header_and_padding(L):
+    for N, K in ((3072, 1024), (4096, 4096), (1024, 4096), (14336, 4096), (4096, 14336), (8192, 28672)):
+        got = binding.packed_size(N, K)
+        assert got == pf.layout(N, K)["total"]
+        assert got == pf.HEADER_BYTES + pf.memory_formula_bits(N, K) // 8      # K % 1024 == 0: no padding
+    # K not a multiple of 1024 pads the code and scale regions to the next multiple
+    assert binding.packed_size(7, 1152) == 256 + 7 * 2048 // 2 + 4 * 7 * 16
+    for bad in ((0, 128), (4, 0), (4, 100), (-1, 128)):
+        assert binding.packed_size(*bad) == 0
+    assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 64, 1))) == 0
+    assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 128, 2))) == 0
+
+
+def test_parse_header_accepts_reference_blob_and_rejects_damage(L):
+    c = make_case(3, 1152, seed=2)
+    blob = pf.pack_reference(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+    assert binding.ptqtp_parse_header(bytes(blob[:256])) == (3, 1152)
+    bad = blob[:256].copy()
+    bad[0] ^= 1
+    with pytest.raises(binding.PtqtpError) as e:
+        binding.ptqtp_parse_header(bytes(bad))
+    assert e.value.status == binding.ERR_FORMAT
+    bad = blob[:256].copy()
+    bad[16] += 1          # N no longer matches the recorded offsets
+    with pytest.raises(binding.PtqtpError):
+        binding.ptqtp_parse_header(bytes(bad))
+    with pytest.raises(binding.PtqtpError) as e:
+        binding.ptqtp_parse_header(bytes(blob[:16]))
+    assert e.value.status == binding.ERR_SIZE
+
+
+def test_host_side_validation_codes(L):
+    shape = binding.make_shape(8, 256)
+    sp = ctypes.byref(shape)
+    ok_ptr = ctypes.c_void_p(0x10000)           # never dereferenced: validation fails first
+    odd_ptr = ctypes.c_void_p(0x10008)
+    size = binding.packed_size(8, 256)
+    assert L.ptqtp_gemv(sp, None, size, ok_ptr, ok_ptr, None) == binding.ERR_NULL
+    assert L.ptqtp_gemv(sp, ok_ptr, size, None, ok_ptr, None) == binding.ERR_NULL
+    assert L.ptqtp_gemv(None, ok_ptr, size, ok_ptr, ok_ptr, None) == binding.ERR_NULL
+    assert L.ptqtp_gemv(sp, odd_ptr, size, ok_ptr, ok_ptr, None) == binding.ERR_ALIGN
+    assert L.ptqtp_gemv(sp, ok_ptr, size, odd_ptr, ok_ptr, None) == binding.ERR_ALIGN
+    assert L.ptqtp_gemv(sp, ok_ptr, size - 1, ok_ptr, ok_ptr, None) == binding.ERR_SIZE
+    bad = binding.make_shape(8, 200)
+    assert L.ptqtp_gemv(ctypes.byref(bad), ok_ptr, size, ok_ptr, ok_ptr, None) == binding.ERR_SHAPE
+    assert L.ptqtp_gemm_skinny(sp, ok_ptr, size, 0, ok_ptr, ok_ptr, None) == binding.ERR_SHAPE
+    assert L.ptqtp_gemm_skinny(sp, ok_ptr, size, 65, ok_ptr, ok_ptr, None) == binding.ERR_SHAPE
+    assert L.ptqtp_gemv_cfg(sp, ok_ptr, size, ok_ptr, ok_ptr, -1, 0, 0, 0, -1, None) == binding.ERR_CONFIG
+    assert L.ptqtp_pack(sp, ok_ptr, ok_ptr, ok_ptr, None, ok_ptr, size, None, None) == binding.ERR_NULL
+    assert L.ptqtp_pack(sp, ok_ptr, odd_ptr, ok_ptr, ok_ptr, ok_ptr, size, None, None) == binding.ERR_ALIGN
+    assert L.ptqtp_unpack(sp, ok_ptr, size - 4, ok_ptr, ok_ptr, ok_ptr, ok_ptr, None, None) == binding.ERR_SIZE
+    assert L.ptqtp_gemv_host(sp, ok_ptr, size, None, ok_ptr, ok_ptr, ok_ptr, None) == binding.ERR_NULL
+
+
+def test_status_strings(L):
+    seen = set()
+    for code in range(0, -9, -1):
+        s = binding.status_string(code)
+        assert s and s != "unknown status"
+        seen.add(s)
+    assert len(seen) == 9
+    assert binding.status_string(-99) == "unknown status"
+
+
+def test_binding_refuses_cpu_tensors(L):
+    import torch
+    with pytest.raises(TypeError):
+        binding.ptqtp_gemv(torch.zeros(binding.packed_size(8, 128), dtype=torch.uint8), 8, 128,
+                           torch.zeros(128, dtype=torch.float16))
+
+
+def test_reference_format_roundtrip_and_damage_detection():
+    c = make_case(6, 1280, seed=3)
+    blob = pf.pack_reference(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+    t1, t2, a1, a2 = pf.unpack_reference(blob)
+    assert np.array_equal(t1, c["T1"]) and np.array_equal(t2, c["T2"])
+    assert np.array_equal(a1.view(np.uint16), c["alpha1"].view(np.uint16))
+    assert np.array_equal(a2.view(np.uint16), c["alpha2"].view(np.uint16))
+    # one trit, one bit position: column 37 of row 2, plane 2 -> lane block 1, e = 5, word 2, bits 10..11
+    c["T2"][2, 37] = -1
+    b2 = pf.pack_reference(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+    off = 256 + (2 * 2 + 0) * 512 + 1 * 16 + 2 * 4
+    word = int.from_bytes(bytes(b2[off:off + 4]), "little")
+    assert (word >> 10) & 3 == 0
+    bad = blob.copy()
+    bad[256] |= 3                       # code 3 does not exist
+    with pytest.raises(ValueError):
+        pf.unpack_reference(bad)

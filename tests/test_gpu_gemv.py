@@ -1,0 +1,206 @@
+"""GPU parity of ptqtp_gemv / ptqtp_gemm_skinny / ptqtp_gemv_host against the fp64 oracle.
+
+Bar: rel-L2 <= 1e-3 and max-abs <= 2e-3 * ||x||_inf * sqrt(K) per batch row (both against the
+fp64 result on the same fp16 inputs)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle.layer import layer_fp64
+from paper_2509_16989_b200 import binding
+from paper_2509_16989_b200.inputs import (LLAMA3_70B, LLAMA3_8B_UNIQUE, QWEN3_0P6B_UP, make_activations,
+                                          make_case, make_weights)
+from gpu_util import assert_parity, dev, oracle_y, pack_case
+
+pytestmark = pytest.mark.gpu
+
+
+def run_gemv(c, **cfg):
+    packed = pack_case(c)
+    if cfg:
+        y = binding.ptqtp_gemv_cfg(packed, c["N"], c["K"], dev(c["x"]), **cfg)
+    else:
+        y = binding.ptqtp_gemv(packed, c["N"], c["K"], dev(c["x"]))
+    torch.cuda.synchronize()
+    return y.cpu().numpy()
+
+
+@pytest.mark.parametrize("N,K", [(1, 128), (2, 256), (3, 1024), (5, 1152), (31, 2048), (33, 3200),
+                                 (130, 4096), (257, 5120), (64, 14336)])
+def test_small_and_ragged_shapes(N, K):
+    c = make_case(N, K, seed=100 + N)
+    assert_parity(run_gemv(c), oracle_y(c), c["x"], "N=%d K=%d" % (N, K))
+
+
+@pytest.mark.parametrize("R,D", [(1, 2), (1, 4), (1, 8), (2, 1), (2, 2), (2, 4), (4, 1), (4, 2)])
+@pytest.mark.parametrize("WS", [1, 2, 4, 8])
+def test_every_launch_configuration(R, D, WS):
+    for N, K in ((67, 8192), (1000, 16384)):
+        c = make_case(N, K, seed=R * 10 + WS)
+        ref = oracle_y(c)
+        packed = pack_case(c)
+        for arith in (0, 1, 2):
+            y = binding.ptqtp_gemv_cfg(packed, N, K, dev(c["x"]), rows_per_warp=R, k_split=WS, ctas_per_sm=1,
+                                       depth=D, arith=arith)
+            torch.cuda.synchronize()
+            assert_parity(y.cpu().numpy(), ref, c["x"], "R=%d WS=%d D=%d arith=%d N=%d K=%d" % (R, WS, D, arith, N, K))
+
+
+def test_k_split_must_divide_the_slices():
+    c = make_case(8, 3072, seed=1)
+    packed = pack_case(c)
+    with pytest.raises(binding.PtqtpError) as e:
+        binding.ptqtp_gemv_cfg(packed, 8, 3072, dev(c["x"]), rows_per_warp=1, k_split=2, depth=2)
+    assert e.value.status == binding.ERR_CONFIG
+
+
+def test_unsupported_configuration_is_rejected():
+    c = make_case(8, 1024, seed=1)
+    packed = pack_case(c)
+    with pytest.raises(binding.PtqtpError) as e:
+        binding.ptqtp_gemv_cfg(packed, 8, 1024, dev(c["x"]), rows_per_warp=3, k_split=1)
+    assert e.value.status == binding.ERR_CONFIG
+
+
+def test_config0_qwen3_up_proj():
+    N, K = QWEN3_0P6B_UP
+    c = make_case(N, K, seed=0)
+    assert_parity(run_gemv(c), oracle_y(c), c["x"], "qwen3 up")
+
+
+@pytest.mark.parametrize("name", sorted(LLAMA3_8B_UNIQUE))
+def test_config1_llama3_8b_shapes_full_size(name):
+    N, K = LLAMA3_8B_UNIQUE[name]
+    c = make_case(N, K, seed=sorted(LLAMA3_8B_UNIQUE).index(name))
+    assert_parity(run_gemv(c), oracle_y(c), c["x"], name)
+
+
+@pytest.mark.parametrize("name", sorted(LLAMA3_70B))
+def test_config3_llama3_70b_shapes_half_zero_planes(name):
+    N, K = LLAMA3_70B[name]
+    c = make_case(N, K, seed=3, p_zero=0.5)
+    y = run_gemv(c)
+    rows = np.unique(np.concatenate([np.arange(0, 64), np.arange(N - 64, N),
+                                     np.random.default_rng(0).integers(0, N, 1024)]))
+    assert_parity(y[rows], oracle_y(c, rows), c["x"], name)
+    assert np.all(np.isfinite(y))
+
+
+def test_special_planes_closed_forms():
+    N, K = 96, 2048
+    c = make_case(N, K, seed=4)
+    x64 = c["x"].astype(np.float64)
+    # all-zero planes -> zero up to the fp32 rounding of (sum of x) - (sum of x)
+    z = np.zeros_like(c["T1"])
+    c0 = dict(c, T1=z, T2=z)
+    assert np.all(np.abs(run_gemv(c0).astype(np.float64)) <= 1e-6)
+    # T1 = -T2 with equal scales -> cancels to (nearly) zero: bounded by the fp32 epilogue rounding
+    cc = dict(c, T2=-c["T1"], alpha2=c["alpha1"])
+    y = run_gemv(cc).astype(np.float64)
+    scale = np.abs(layer_fp64(c["T1"], z, c["alpha1"], c["alpha2"], c["x"]))
+    assert np.all(np.abs(y) <= 2e-3 * scale.max())
+    # one +1 per row, alpha1 = 1 -> gather of x (exact: a single term)
+    cols = np.random.default_rng(1).integers(0, K, N)
+    T1 = np.zeros_like(c["T1"])
+    T1[np.arange(N), cols] = 1
+    ones = np.ones_like(c["alpha1"])
+    cg = dict(c, T1=T1, T2=z, alpha1=ones, alpha2=ones)
+    yg = run_gemv(cg).astype(np.float64)
+    assert np.allclose(yg, x64[cols], rtol=2e-3, atol=2e-3)
+    # all +1 in plane 1 -> y_i = sum_g alpha1[i,g] * (group sums of x)
+    cp = dict(c, T1=np.ones_like(c["T1"]), T2=z)
+    assert_parity(run_gemv(cp), oracle_y(cp), c["x"], "all +1")
+    cm = dict(c, T1=-np.ones_like(c["T1"]), T2=np.ones_like(c["T1"]))
+    assert_parity(run_gemv(cm), oracle_y(cm), c["x"], "all -1 / +1")
+
+
+@pytest.mark.parametrize("scale", [2.0 ** -12, 2.0 ** -6, 1.0, 2.0 ** 6, 2.0 ** 11])
+def test_activation_dynamic_range(scale):
+    c = make_case(128, 4096, seed=6)
+    c["x"] = (c["x"].astype(np.float32) * scale).astype(np.float16)
+    assert_parity(run_gemv(c), oracle_y(c), c["x"], "scale %g" % scale)
+
+
+def test_activations_with_outliers_zero_blocks_and_negative_scales():
+    c = make_case(128, 4096, seed=7)
+    x = c["x"].astype(np.float32)
+    x[::97] *= 50.0                 # heavy outliers
+    x[1024:1056] = 0.0              # an all-zero lane block
+    x[2048:2176] = 0.0              # an all-zero group
+    x[5] = 6.0e4                    # close to the fp16 maximum
+    x[40] = 6.0e-8                  # fp16 subnormal
+    c["x"] = x.astype(np.float16)
+    c["alpha2"] = (-c["alpha2"].astype(np.float32)).astype(np.float16)
+    c["alpha1"][::3, ::2] = 0
+    assert_parity(run_gemv(c), oracle_y(c), c["x"], "outliers")
+
+
+def test_output_guard_bands_and_determinism():
+    c = make_case(77, 3072, seed=8)
+    packed = pack_case(c)
+    buf = torch.full((77 + 64,), float("nan"), dtype=torch.float16, device="cuda")
+    y = buf[32:32 + 77]
+    # y must be 16-byte aligned: 32 halves = 64 bytes
+    binding.ptqtp_gemv(packed, 77, 3072, dev(c["x"]), y=y)
+    torch.cuda.synchronize()
+    host = buf.cpu().numpy()
+    assert np.all(np.isnan(host[:32])) and np.all(np.isnan(host[32 + 77:]))
+    first = host[32:32 + 77].copy()
+    for _ in range(3):
+        again = binding.ptqtp_gemv(packed, 77, 3072, dev(c["x"])).cpu().numpy()
+        assert np.array_equal(again.view(np.uint16), first.view(np.uint16))
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 8, 17, 64])
+def test_gemm_skinny_matches_oracle_per_row(M):
+    c = make_case(192, 3072, seed=20 + M, M=M)
+    packed = pack_case(c)
+    X = dev(np.atleast_2d(c["x"]))
+    Y = binding.ptqtp_gemm_skinny(packed, 192, 3072, X)
+    torch.cuda.synchronize()
+    assert Y.shape == (M, 192)
+    ref = np.atleast_2d(oracle_y(c))
+    assert_parity(Y.cpu().numpy(), ref, np.atleast_2d(c["x"]), "M=%d" % M)
+
+
+def test_gemm_skinny_config2_shape_batch8_sampled_rows():
+    N, K = LLAMA3_8B_UNIQUE["gate_up"]
+    c = make_case(N, K, seed=2, M=8)
+    packed = pack_case(c)
+    Y = binding.ptqtp_gemm_skinny(packed, N, K, dev(c["x"]))
+    torch.cuda.synchronize()
+    rows = np.unique(np.random.default_rng(5).integers(0, N, 2048))
+    assert_parity(Y.cpu().numpy()[:, rows], oracle_y(c, rows), c["x"], "gate_up M=8")
+
+
+def test_gemv_host_entry_point():
+    c = make_case(300, 2048, seed=9)
+    packed = pack_case(c)
+    x_host = torch.from_numpy(c["x"]).pin_memory()
+    y_host = torch.empty(300, dtype=torch.float16).pin_memory()
+    x_dev = torch.empty(2048, dtype=torch.float16, device="cuda")
+    y_dev = torch.empty(300, dtype=torch.float16, device="cuda")
+    binding.ptqtp_gemv_host(packed, 300, 2048, x_host, y_host, x_dev, y_dev)
+    torch.cuda.synchronize()
+    assert_parity(y_host.numpy(), oracle_y(c), c["x"], "host call")
+    assert np.array_equal(y_host.numpy().view(np.uint16), y_dev.cpu().numpy().view(np.uint16))
+
+
+def test_decomposed_weights_end_to_end():
+    # realistic-weight path: W -> oracle decomposition -> pack -> GEMV; parity against the oracle's
+    # layer product on the decomposed planes, and the reconstruction error in its expected range.
+    from oracle.c_oracle import decompose_c
+    from oracle.decompose import reconstruction_error
+    N, K = 512, 4096
+    W = make_weights(N, K, seed=40)
+    d = decompose_c(W)
+    c = dict(N=N, K=K, T1=d["T1"], T2=d["T2"], alpha1=d["alpha1_fp16"], alpha2=d["alpha2_fp16"],
+             x=make_activations(K, seed=41))
+    y = run_gemv(c)
+    assert_parity(y, oracle_y(c), c["x"], "decomposed")
+    err = reconstruction_error(W, d["T1"], d["T2"], d["alpha1_fp16"], d["alpha2_fp16"])
+    assert 0.10 < err < 0.25
+    # and against the unquantised layer: the quantisation error dominates, at about that level
+    dense = W.astype(np.float64) @ c["x"].astype(np.float64)
+    rel = np.linalg.norm(y.astype(np.float64) - dense) / np.linalg.norm(dense)
+    assert rel < 2.5 * err
