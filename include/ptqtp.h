@@ -41,6 +41,25 @@
  *                       padding groups are zero.
  *   ptqtp_packed_size = 256 + N*K_pad/2 + 4*N*K_pad/128 bytes, i.e. the Appendix B figure
  *   2*N*K*2 + (K/128)*2*N*16 bits plus the header and the K padding.
+ *
+ * Packed format 2 (same storage model; laid out for integer dot products: one mask yields four
+ * byte-sized codes of four consecutive columns, see ptqtp_gemv):
+ *   [0, 256)            header as above with format(2); the K_pad slot holds 2048 * ceil(K/2048) and the
+ *                       scales_offset slot holds the row-pair stride in bytes.
+ *   body  (at 256)      ceil(N/2) row pairs, row pair p = rows 2p and 2p+1 (a missing row 2p+1 is stored
+ *                       as trit 0 with scales 0).  A row pair is a strip of ceil(K/2048) slice units, slice s
+ *                       covering columns 2048 s .. min(K, 2048 (s+1)) - 1 with A = columns/64 lane blocks:
+ *                         codes   4 * A atoms of 16 bytes; atom (i, l), i = 0..3, l = 0..A-1, at byte
+ *                                 16 * (i * A + l), covers the 16 columns 2048 s + 64 l + 16 i + e, e = 0..15,
+ *                                 one byte per column (byte e): bits [1:0] = code of (row 2p, plane 1),
+ *                                 [3:2] = (row 2p, plane 2), [5:4] = (row 2p+1, plane 1),
+ *                                 [7:6] = (row 2p+1, plane 2); code q = trit + 1 in {0,1,2}.
+ *                         scales  A/2 quads of 8 bytes at byte 64 * A, one per 128-column group in column
+ *                                 order: fp16 alpha1[2p], alpha2[2p], alpha1[2p+1], alpha2[2p+1].
+ *                         the unit is zero-padded to a multiple of 16 bytes (only when K/128 is odd).
+ *                       A full slice unit is 2048 + 128 = 2176 bytes.
+ *   ptqtp_packed_size = 256 + ceil(N/2) * (K + K/16 rounded up per unit) bytes; for even N and K % 256 == 0
+ *   exactly the Appendix B figure plus the header.
  */
 #ifndef PTQTP_H
 #define PTQTP_H
@@ -74,11 +93,12 @@ typedef struct {
     int32_t n_out;   /* N: output features (rows of W)            */
     int32_t k_in;    /* K: input features, multiple of 128        */
     int32_t group;   /* scale group size along K; must be 128     */
-    int32_t format;  /* packed format id; must be 1               */
+    int32_t format;  /* packed format id: 1 or 2                  */
 } ptqtp_shape;
 
 #define PTQTP_GROUP 128
 #define PTQTP_FORMAT_V1 1
+#define PTQTP_FORMAT_V2 2
 #define PTQTP_HEADER_BYTES 256
 #define PTQTP_MAX_BATCH 64
 
@@ -106,8 +126,11 @@ PTQTP_API ptqtp_status ptqtp_unpack(const ptqtp_shape *shape /* host */, const v
  * Sec. 4: additions/subtractions of x, one scale multiply per group and plane).
  * packed: device blob from ptqtp_pack (its header is not re-read; `shape` is trusted);
  * x: device fp16 [K]; y: device fp16 [N], fully overwritten.  x and y must not alias packed.
- * Arithmetic: fp16 x, short fp16 partial sums flushed into fp32 accumulators, fp32 scale
- * epilogue, one rounding to fp16 at the store.  Non-finite x gives unspecified non-finite y. */
+ * Arithmetic, format 1: fp16 x times codes, fp32 accumulators, fp32 scale epilogue.
+ * Arithmetic, format 2: x is turned into 16-bit block fixed point per 64 columns (exact for values within
+ * 2^-5 of the block maximum, otherwise rounded to 2^-16 of it), sign-select sums are exact int32, the
+ * scale epilogue and the sums over groups are fp32.  One rounding to fp16 at the store in both.
+ * Non-finite x gives unspecified y. */
 PTQTP_API ptqtp_status ptqtp_gemv(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                         const uint16_t *x, uint16_t *y, void *stream);
 
@@ -131,7 +154,10 @@ PTQTP_API ptqtp_status ptqtp_gemv_host(const ptqtp_shape *shape /* host */, cons
  * every combination with rows_per_warp is built); 0 in any of these selects the library's own choice.
  * arith: accumulation of the sign-selected activations -- 0 = fp32 accumulator fed by mixed-precision
  * FMAs (fp16 operands), 1 = fp16x2 chains of 4 flushed into fp32, 2 = chains of 8, -1 = library choice.
- * PTQTP_ERR_CONFIG if the combination is not built. */
+ * PTQTP_ERR_CONFIG if the combination is not built.
+ * For a format-2 blob the arguments mean: rows_per_warp must be 0; k_split = warps per CTA (1..16, 0 = auto);
+ * ctas_per_sm must be 0 or 1 (one persistent CTA per SM); depth = slice units in flight per warp
+ * (2, 3, 4, 6, 8; 0 = auto); arith must be -1 or 3 (integer dot products). */
 PTQTP_API ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                             const uint16_t *x, uint16_t *y, int32_t rows_per_warp, int32_t k_split,
                             int32_t ctas_per_sm, int32_t depth, int32_t arith, void *stream);

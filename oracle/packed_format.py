@@ -13,6 +13,17 @@ one fp16 scale per plane per 128-column group):
   scales           for each row i, for each group g < K_pad/128: u16 alpha1 bits, u16 alpha2 bits
                    (zero for padding groups).
 
+Format 2 (same header with format = 2; the K_pad slot holds 2048 * ceil(K/2048), the scales-offset slot the
+row-pair stride in bytes):
+
+  body             for each row pair p (rows 2p, 2p+1; a missing odd row counts as trit 0, scales 0), for each
+                   slice s of up to 2048 columns with A = columns/64 lane blocks: 4*A atoms of 16 bytes, atom
+                   (i, l) at byte 16*(i*A + l) holding columns 2048 s + 64 l + 16 i + e (e = 0..15), one byte
+                   per column = code(2p, plane 1) | code(2p, plane 2) << 2 | code(2p+1, plane 1) << 4
+                   | code(2p+1, plane 2) << 6; then A/2 quads of 4 little-endian u16 (alpha1[2p], alpha2[2p],
+                   alpha1[2p+1], alpha2[2p+1]) for the slice's 128-column groups; then zero padding to a
+                   multiple of 16 bytes.
+
 Written independently of the CUDA pack/unpack kernels (plain numpy bit operations) so that the two
 can be compared byte for byte.
 """
@@ -120,3 +131,98 @@ def unpack_reference(blob):
     a1 = sc[:, :K // 128, 0].copy().view(np.float16)
     a2 = sc[:, :K // 128, 1].copy().view(np.float16)
     return planes[0], planes[1], a1, a2
+
+
+# ----------------------------------------------------------------------------- format 2
+def layout_v2(N, K):
+    if N <= 0 or K <= 0 or K % 128:
+        raise ValueError("N > 0 and K a positive multiple of 128 required")
+    nrp = (N + 1) // 2
+    slices = (K + 2047) // 2048
+    units = []                                   # (first column, columns, byte offset in the strip, bytes)
+    off = 0
+    for sl in range(slices):
+        cols = min(2048, K - 2048 * sl)
+        size = -(-(cols + cols // 16) // 16) * 16
+        units.append((2048 * sl, cols, off, size))
+        off += size
+    return dict(N=N, K=K, nrp=nrp, slices=slices, units=units, strip=off, codes_off=HEADER_BYTES,
+                total=HEADER_BYTES + nrp * off)
+
+
+def pack_reference_v2(T1, T2, alpha1, alpha2):
+    """Planes int8 [N,K], scales fp16 [N,K/128] -> format-2 blob (numpy uint8)."""
+    T1 = np.asarray(T1, dtype=np.int8)
+    T2 = np.asarray(T2, dtype=np.int8)
+    N, K = T1.shape
+    L = layout_v2(N, K)
+    if np.any(np.abs(T1) > 1) or np.any(np.abs(T2) > 1):
+        raise ValueError("trit out of range")
+    nrp = L["nrp"]
+    q = np.ones((2, 2 * nrp, K), dtype=np.uint8)                  # [plane, row, column]; a missing row is trit 0
+    q[0, :N] = (T1.astype(np.int16) + 1).astype(np.uint8)
+    q[1, :N] = (T2.astype(np.int16) + 1).astype(np.uint8)
+    col_byte = (q[0, 0::2] | (q[1, 0::2] << 2) | (q[0, 1::2] << 4) | (q[1, 1::2] << 6)).astype(np.uint8)
+    sc = np.zeros((2 * nrp, K // 128, 2), dtype="<u2")             # [row, group, plane]
+    sc[:N, :, 0] = np.asarray(alpha1, dtype=np.float16).view(np.uint16)
+    sc[:N, :, 1] = np.asarray(alpha2, dtype=np.float16).view(np.uint16)
+    quads = np.concatenate([sc[0::2], sc[1::2]], axis=2)           # [row pair, group, 4]
+    blob = np.zeros(L["total"], dtype=np.uint8)
+    hdr = MAGIC + struct.pack("<IIiiiiQQQ", 1, 2, N, K, 128, 2048 * L["slices"], L["codes_off"], L["strip"],
+                              L["total"])
+    blob[:len(hdr)] = np.frombuffer(hdr, dtype=np.uint8)
+    body = blob[L["codes_off"]:].reshape(nrp, L["strip"])
+    for c0, cols, off, size in L["units"]:
+        A = cols // 64
+        atoms = col_byte[:, c0:c0 + cols].reshape(nrp, A, 4, 16)   # [row pair, lane block, i, e]
+        body[:, off:off + 4 * A * 16] = atoms.transpose(0, 2, 1, 3).reshape(nrp, -1)
+        g0 = c0 // 128
+        body[:, off + 64 * A:off + 64 * A + 4 * A] = (
+            np.ascontiguousarray(quads[:, g0:g0 + A // 2]).reshape(nrp, -1).view(np.uint8))
+    return blob
+
+
+def unpack_reference_v2(blob):
+    """Format-2 blob (numpy uint8) -> T1, T2 int8 [N,K], alpha1, alpha2 fp16 [N,K/128]."""
+    blob = np.asarray(blob, dtype=np.uint8)
+    hdr = bytes(blob[:HEADER_BYTES])
+    if hdr[:8] != MAGIC:
+        raise ValueError("bad magic")
+    version, fmt, N, K, group, K_pad, codes_off, stride, total = struct.unpack("<IIiiiiQQQ", hdr[8:56])
+    if version != 1 or fmt != 2 or group != 128 or any(hdr[56:]):
+        raise ValueError("bad version/format/group")
+    L = layout_v2(N, K)
+    if (K_pad, codes_off, stride, total) != (2048 * L["slices"], L["codes_off"], L["strip"], L["total"]):
+        raise ValueError("header inconsistent with its shape")
+    if blob.size < L["total"]:
+        raise ValueError("blob too small")
+    nrp = L["nrp"]
+    body = blob[L["codes_off"]:L["total"]].reshape(nrp, L["strip"])
+    col_byte = np.zeros((nrp, K), dtype=np.uint8)
+    quads = np.zeros((nrp, K // 128, 4), dtype="<u2")
+    for c0, cols, off, size in L["units"]:
+        A = cols // 64
+        atoms = body[:, off:off + 4 * A * 16].reshape(nrp, 4, A, 16)
+        col_byte[:, c0:c0 + cols] = atoms.transpose(0, 2, 1, 3).reshape(nrp, cols)
+        g0 = c0 // 128
+        quads[:, g0:g0 + A // 2] = np.ascontiguousarray(body[:, off + 64 * A:off + 68 * A]).view("<u2").reshape(
+            nrp, A // 2, 4)
+        if np.any(body[:, off + 68 * A:off + size] != 0):
+            raise ValueError("unit padding must be zero")
+    planes = []
+    for plane in range(2):
+        t = np.zeros((2 * nrp, K), dtype=np.int16)
+        for r in range(2):
+            code = (col_byte >> (4 * r + 2 * plane)) & 3
+            if np.any(code == 3):
+                raise ValueError("code 3 found")
+            t[r::2] = code.astype(np.int16) - 1
+        if 2 * nrp > N and np.any(t[N:] != 0):
+            raise ValueError("the missing odd row must hold trit 0")
+        planes.append(t[:N].astype(np.int8))
+    if 2 * nrp > N and np.any(quads[-1, :, 2:] != 0):
+        raise ValueError("the missing odd row must have zero scales")
+    a1 = np.zeros((2 * nrp, K // 128), dtype=np.uint16)
+    a2 = np.zeros((2 * nrp, K // 128), dtype=np.uint16)
+    a1[0::2], a2[0::2], a1[1::2], a2[1::2] = quads[:, :, 0], quads[:, :, 1], quads[:, :, 2], quads[:, :, 3]
+    return planes[0], planes[1], a1[:N].view(np.float16), a2[:N].view(np.float16)

@@ -13,6 +13,8 @@ LIB_PATH = os.path.join(_HERE, "libptqtp.so")
 
 GROUP = 128
 FORMAT_V1 = 1
+FORMAT_V2 = 2
+DEFAULT_FORMAT = FORMAT_V2
 HEADER_BYTES = 256
 MAX_BATCH = 64
 
@@ -77,12 +79,14 @@ def status_string(status):
     return lib().ptqtp_status_string(int(status)).decode()
 
 
-def make_shape(N, K, group=GROUP, fmt=FORMAT_V1):
+def make_shape(N, K, group=GROUP, fmt=None):
+    if fmt is None:
+        fmt = DEFAULT_FORMAT
     return Shape(int(N), int(K), int(group), int(fmt))
 
 
-def packed_size(N, K):
-    return int(lib().ptqtp_packed_size(ctypes.byref(make_shape(N, K))))
+def packed_size(N, K, fmt=None):
+    return int(lib().ptqtp_packed_size(ctypes.byref(make_shape(N, K, fmt=fmt))))
 
 
 def _stream_ptr(stream):
@@ -102,11 +106,11 @@ def _check(status, what):
         raise PtqtpError(status, what)
 
 
-def ptqtp_pack(T1, T2, alpha1, alpha2, packed=None, dev_status=None, stream=None):
+def ptqtp_pack(T1, T2, alpha1, alpha2, packed=None, dev_status=None, stream=None, fmt=None):
     """Pack int8 planes [N,K] and fp16 scales [N,K/128] (CUDA tensors).  Returns (packed uint8 tensor, dev_status)."""
     N, K = T1.shape
-    shape = make_shape(N, K)
-    nbytes = packed_size(N, K)
+    shape = make_shape(N, K, fmt=fmt)
+    nbytes = packed_size(N, K, fmt=fmt)
     if nbytes == 0:
         raise PtqtpError(ERR_SHAPE, "ptqtp_packed_size")
     if packed is None:
@@ -121,9 +125,9 @@ def ptqtp_pack(T1, T2, alpha1, alpha2, packed=None, dev_status=None, stream=None
     return packed, dev_status
 
 
-def ptqtp_unpack(packed, N, K, dev_status=None, stream=None):
+def ptqtp_unpack(packed, N, K, dev_status=None, stream=None, fmt=None):
     """Inverse of ptqtp_pack.  Returns (T1, T2, alpha1, alpha2, dev_status) as CUDA tensors."""
-    shape = make_shape(N, K)
+    shape = make_shape(N, K, fmt=fmt)
     dev = packed.device
     T1 = torch.empty((N, K), dtype=torch.int8, device=dev)
     T2 = torch.empty((N, K), dtype=torch.int8, device=dev)
@@ -139,9 +143,9 @@ def ptqtp_unpack(packed, N, K, dev_status=None, stream=None):
     return T1, T2, a1, a2, dev_status
 
 
-def ptqtp_gemv(packed, N, K, x, y=None, stream=None):
+def ptqtp_gemv(packed, N, K, x, y=None, stream=None, fmt=None):
     """y[N] = layer(x[K]) from a packed blob; fp16 CUDA tensors."""
-    shape = make_shape(N, K)
+    shape = make_shape(N, K, fmt=fmt)
     if y is None:
         y = torch.empty(N, dtype=torch.float16, device=x.device)
     st = lib().ptqtp_gemv(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
@@ -151,8 +155,8 @@ def ptqtp_gemv(packed, N, K, x, y=None, stream=None):
 
 
 def ptqtp_gemv_cfg(packed, N, K, x, y=None, rows_per_warp=0, k_split=0, ctas_per_sm=0, depth=0, arith=-1,
-                   stream=None):
-    shape = make_shape(N, K)
+                   stream=None, fmt=None):
+    shape = make_shape(N, K, fmt=fmt)
     if y is None:
         y = torch.empty(N, dtype=torch.float16, device=x.device)
     st = lib().ptqtp_gemv_cfg(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
@@ -163,9 +167,9 @@ def ptqtp_gemv_cfg(packed, N, K, x, y=None, rows_per_warp=0, k_split=0, ctas_per
     return y
 
 
-def ptqtp_gemm_skinny(packed, N, K, X, Y=None, stream=None):
+def ptqtp_gemm_skinny(packed, N, K, X, Y=None, stream=None, fmt=None):
     """Y[M,N] = layer applied to each row of X[M,K]; fp16 CUDA tensors, 1 <= M <= 64."""
-    shape = make_shape(N, K)
+    shape = make_shape(N, K, fmt=fmt)
     M = X.shape[0]
     if Y is None:
         Y = torch.empty((M, N), dtype=torch.float16, device=X.device)
@@ -176,9 +180,9 @@ def ptqtp_gemm_skinny(packed, N, K, X, Y=None, stream=None):
     return Y
 
 
-def ptqtp_gemv_host(packed, N, K, x_host, y_host, x_dev, y_dev, stream=None):
+def ptqtp_gemv_host(packed, N, K, x_host, y_host, x_dev, y_dev, stream=None, fmt=None):
     """Host-buffer call: H2D copy of x, GEMV, D2H copy of y, all on `stream` (no sync)."""
-    shape = make_shape(N, K)
+    shape = make_shape(N, K, fmt=fmt)
     for t, what in ((x_host, "x_host"), (y_host, "y_host")):
         if t.is_cuda or t.dtype != torch.float16 or not t.is_contiguous():
             raise TypeError("%s must be a contiguous fp16 host tensor" % what)
@@ -191,9 +195,9 @@ def ptqtp_gemv_host(packed, N, K, x_host, y_host, x_dev, y_dev, stream=None):
 
 
 def ptqtp_parse_header(header_bytes):
-    """Parse a host copy (bytes) of a blob's header; returns (N, K)."""
+    """Parse a host copy (bytes) of a blob's header; returns (N, K, format)."""
     buf = ctypes.create_string_buffer(bytes(header_bytes), len(header_bytes))
     shape = Shape()
     st = lib().ptqtp_parse_header(ctypes.cast(buf, ctypes.c_void_p), len(header_bytes), ctypes.byref(shape))
     _check(st, "ptqtp_parse_header")
-    return shape.n_out, shape.k_in
+    return shape.n_out, shape.k_in, shape.format

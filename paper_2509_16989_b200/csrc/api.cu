@@ -31,13 +31,30 @@ int sm_count() {
     return cached;
 }
 
-static ptqtp_status check_packed(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, Layout* L) {
+// Layout of either format, as selected by shape->format.
+struct AnyLayout {
+    bool v2;
+    Layout l1;
+    Layout2 l2;
+};
+
+static ptqtp_status check_packed(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, AnyLayout* L) {
     if (!shape || !packed) return PTQTP_ERR_NULL;
     if (!shape_ok(shape)) return PTQTP_ERR_SHAPE;
-    *L = make_layout(shape);
+    L->v2 = shape->format == PTQTP_FORMAT_V2;
+    if (L->v2) L->l2 = make_layout2(shape); else L->l1 = make_layout(shape);
     if (!aligned16(packed)) return PTQTP_ERR_ALIGN;
-    if (packed_bytes < L->total) return PTQTP_ERR_SIZE;
+    if (packed_bytes < packed_total(shape)) return PTQTP_ERR_SIZE;
     return PTQTP_OK;
+}
+
+static ptqtp_status gemv_any(const AnyLayout& L, const void* packed, const uint16_t* x, uint16_t* y, int p0, int p1,
+                             int p2, int p3, int p4, cudaStream_t st) {
+    if (L.v2) {
+        if (p0 != 0 || p2 > 1 || (p4 != -1 && p4 != 3)) return PTQTP_ERR_CONFIG;
+        return launch_gemv2(L.l2, packed, x, y, p1, p3, st);
+    }
+    return launch_gemv(L.l1, packed, x, y, p0, p1, p2, p3, p4, st);
 }
 
 }  // namespace ptqtp
@@ -48,43 +65,47 @@ extern "C" {
 
 size_t ptqtp_packed_size(const ptqtp_shape* shape) {
     if (!shape_ok(shape)) return 0;
-    return make_layout(shape).total;
+    return packed_total(shape);
 }
 
 ptqtp_status ptqtp_pack(const ptqtp_shape* shape, const int8_t* T1, const int8_t* T2, const uint16_t* alpha1,
                         const uint16_t* alpha2, void* packed, size_t packed_bytes, int32_t* dev_status,
                         void* stream) {
     if (!T1 || !T2 || !alpha1 || !alpha2) return PTQTP_ERR_NULL;
-    Layout L;
+    AnyLayout L;
     ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
     if (s != PTQTP_OK) return s;
     if (!aligned16(T1) || !aligned16(T2) || !aligned16(alpha1) || !aligned16(alpha2)) return PTQTP_ERR_ALIGN;
     if (dev_status && (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return PTQTP_ERR_ALIGN;
-    return launch_pack(L, T1, T2, alpha1, alpha2, packed, dev_status, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return L.v2 ? launch_pack2(L.l2, T1, T2, alpha1, alpha2, packed, dev_status, st)
+                : launch_pack(L.l1, T1, T2, alpha1, alpha2, packed, dev_status, st);
 }
 
 ptqtp_status ptqtp_unpack(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, int8_t* T1,
                           int8_t* T2, uint16_t* alpha1, uint16_t* alpha2, int32_t* dev_status, void* stream) {
     if (!T1 || !T2 || !alpha1 || !alpha2) return PTQTP_ERR_NULL;
-    Layout L;
+    AnyLayout L;
     ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
     if (s != PTQTP_OK) return s;
     if (!aligned16(T1) || !aligned16(T2) || !aligned16(alpha1) || !aligned16(alpha2)) return PTQTP_ERR_ALIGN;
     if (dev_status && (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return PTQTP_ERR_ALIGN;
-    return launch_unpack(L, packed, T1, T2, alpha1, alpha2, dev_status, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return L.v2 ? launch_unpack2(L.l2, packed, T1, T2, alpha1, alpha2, dev_status, st)
+                : launch_unpack(L.l1, packed, T1, T2, alpha1, alpha2, dev_status, st);
 }
 
 ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, const uint16_t* x,
                             uint16_t* y, int32_t rows_per_warp, int32_t k_split, int32_t ctas_per_sm,
                             int32_t depth, int32_t arith, void* stream) {
     if (!x || !y) return PTQTP_ERR_NULL;
-    Layout L;
+    AnyLayout L;
     ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
     if (s != PTQTP_OK) return s;
     if (!aligned16(x) || !aligned16(y)) return PTQTP_ERR_ALIGN;
     if (rows_per_warp < 0 || k_split < 0 || ctas_per_sm < 0 || depth < 0 || arith < -1) return PTQTP_ERR_CONFIG;
-    return launch_gemv(L, packed, x, y, rows_per_warp, k_split, ctas_per_sm, depth, arith,
-                       static_cast<cudaStream_t>(stream));
+    return gemv_any(L, packed, x, y, rows_per_warp, k_split, ctas_per_sm, depth, arith,
+                    static_cast<cudaStream_t>(stream));
 }
 
 ptqtp_status ptqtp_gemv(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, const uint16_t* x,
@@ -95,28 +116,36 @@ ptqtp_status ptqtp_gemv(const ptqtp_shape* shape, const void* packed, size_t pac
 ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, int32_t m,
                                const uint16_t* X, uint16_t* Y, void* stream) {
     if (!X || !Y) return PTQTP_ERR_NULL;
-    Layout L;
+    AnyLayout L;
     ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
     if (s != PTQTP_OK) return s;
     if (m < 1 || m > PTQTP_MAX_BATCH) return PTQTP_ERR_SHAPE;
     if (!aligned16(X) || !aligned16(Y)) return PTQTP_ERR_ALIGN;
-    return launch_gemm_skinny(L, packed, m, X, Y, static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (L.v2) {
+        for (int i = 0; i < m; ++i) {
+            s = launch_gemv2(L.l2, packed, X + (size_t)i * L.l2.k, Y + (size_t)i * L.l2.n, 0, 0, st);
+            if (s != PTQTP_OK) return s;
+        }
+        return PTQTP_OK;
+    }
+    return launch_gemm_skinny(L.l1, packed, m, X, Y, st);
 }
 
 ptqtp_status ptqtp_gemv_host(const ptqtp_shape* shape, const void* packed, size_t packed_bytes,
                              const uint16_t* x_host, uint16_t* y_host, uint16_t* x_dev, uint16_t* y_dev,
                              void* stream) {
     if (!x_host || !y_host || !x_dev || !y_dev) return PTQTP_ERR_NULL;
-    Layout L;
+    AnyLayout L;
     ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
     if (s != PTQTP_OK) return s;
     if (!aligned16(x_dev) || !aligned16(y_dev)) return PTQTP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)L.k * 2, cudaMemcpyHostToDevice, st);
+    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)shape->k_in * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
-    s = launch_gemv(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
+    s = gemv_any(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
     if (s != PTQTP_OK) return s;
-    e = cudaMemcpyAsync(y_host, y_dev, (size_t)L.n * 2, cudaMemcpyDeviceToHost, st);
+    e = cudaMemcpyAsync(y_host, y_dev, (size_t)shape->n_out * 2, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
     return PTQTP_OK;
 }
@@ -126,13 +155,21 @@ ptqtp_status ptqtp_parse_header(const void* header_host, size_t bytes, ptqtp_sha
     if (bytes < sizeof(Header)) return PTQTP_ERR_SIZE;
     Header h;
     memcpy(&h, header_host, sizeof(Header));
-    if (memcmp(h.magic, "PTQTPB2\0", 8) != 0 || h.version != kVersion || h.format != PTQTP_FORMAT_V1)
+    if (memcmp(h.magic, "PTQTPB2\0", 8) != 0 || h.version != kVersion ||
+        (h.format != PTQTP_FORMAT_V1 && h.format != PTQTP_FORMAT_V2))
         return PTQTP_ERR_FORMAT;
     ptqtp_shape s = {h.n, h.k, h.group, (int32_t)h.format};
     if (!shape_ok(&s)) return PTQTP_ERR_FORMAT;
-    const Layout L = make_layout(&s);
-    if (h.k_pad != L.k_pad || h.codes_off != L.codes_off || h.scales_off != L.scales_off || h.total != L.total)
-        return PTQTP_ERR_FORMAT;
+    if (h.format == PTQTP_FORMAT_V1) {
+        const Layout L = make_layout(&s);
+        if (h.k_pad != L.k_pad || h.codes_off != L.codes_off || h.scales_off != L.scales_off || h.total != L.total)
+            return PTQTP_ERR_FORMAT;
+    } else {
+        const Layout2 L = make_layout2(&s);
+        if (h.k_pad != L.slices * kSlice2 || h.codes_off != L.codes_off || h.scales_off != L.strip ||
+            h.total != L.total)
+            return PTQTP_ERR_FORMAT;
+    }
     *shape = s;
     return PTQTP_OK;
 }

@@ -30,7 +30,7 @@ static_assert(sizeof(Header) <= PTQTP_HEADER_BYTES, "header must fit its slot");
 
 inline bool shape_ok(const ptqtp_shape* s) {
     return s && s->n_out > 0 && s->k_in > 0 && s->group == kGroup && s->k_in % kGroup == 0 &&
-           s->format == PTQTP_FORMAT_V1;
+           (s->format == PTQTP_FORMAT_V1 || s->format == PTQTP_FORMAT_V2);
 }
 
 inline Layout make_layout(const ptqtp_shape* s) {
@@ -44,6 +44,39 @@ inline Layout make_layout(const ptqtp_shape* s) {
     L.scales_off = L.codes_off + (size_t)L.n * L.slices * kChunkBytes;
     L.total = L.scales_off + (size_t)L.n * L.groups_pad * 4;
     return L;
+}
+
+// ---- format 2: row-pair interleaved, 2048-column slices (see ptqtp.h) ----
+constexpr int kSlice2 = 2048;        // input columns per slice of format 2
+constexpr int kLane2 = 64;           // input columns per lane block of format 2
+constexpr int kUnit2 = 2176;         // bytes of a full slice unit: 2048 code bytes + 128 scale bytes
+
+struct Layout2 {
+    int n, k, nrp;                   // rows, columns, row pairs = ceil(n / 2)
+    int slices;                      // ceil(k / 2048)
+    int last_active;                 // 64-column lane blocks in the last slice (1..32)
+    int last_unit;                   // bytes of the last slice's unit (multiple of 16)
+    size_t strip;                    // bytes of one row pair: (slices - 1) * 2176 + last_unit
+    size_t codes_off, total;
+};
+
+inline Layout2 make_layout2(const ptqtp_shape* s) {
+    Layout2 L;
+    L.n = s->n_out;
+    L.k = s->k_in;
+    L.nrp = (s->n_out + 1) / 2;
+    L.slices = (s->k_in + kSlice2 - 1) / kSlice2;
+    const int last_cols = s->k_in - (L.slices - 1) * kSlice2;
+    L.last_active = last_cols / kLane2;
+    L.last_unit = (last_cols + last_cols / 16 + 15) / 16 * 16;
+    L.strip = (size_t)(L.slices - 1) * kUnit2 + L.last_unit;
+    L.codes_off = PTQTP_HEADER_BYTES;
+    L.total = L.codes_off + (size_t)L.nrp * L.strip;
+    return L;
+}
+
+inline size_t packed_total(const ptqtp_shape* s) {
+    return s->format == PTQTP_FORMAT_V2 ? make_layout2(s).total : make_layout(s).total;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -60,6 +93,12 @@ ptqtp_status launch_gemv(const Layout& L, const void* packed, const uint16_t* x,
                          int rows_per_warp, int k_split, int ctas_per_sm, int depth, int arith, cudaStream_t st);
 ptqtp_status launch_gemm_skinny(const Layout& L, const void* packed, int m, const uint16_t* X,
                                 uint16_t* Y, cudaStream_t st);
+ptqtp_status launch_pack2(const Layout2& L, const int8_t* T1, const int8_t* T2, const uint16_t* a1,
+                          const uint16_t* a2, void* packed, int32_t* dev_status, cudaStream_t st);
+ptqtp_status launch_unpack2(const Layout2& L, const void* packed, int8_t* T1, int8_t* T2, uint16_t* a1,
+                            uint16_t* a2, int32_t* dev_status, cudaStream_t st);
+ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
+                          int depth, cudaStream_t st);
 int sm_count();
 
 }  // namespace ptqtp

@@ -14,8 +14,11 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def pack_case(c):
-    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
+FORMATS = (binding.FORMAT_V1, binding.FORMAT_V2)
+
+
+def pack_case(c, fmt=None):
+    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=fmt)
     torch.cuda.synchronize()
     assert int(st.item()) == 0
     return packed

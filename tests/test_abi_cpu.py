@@ -36,21 +36,32 @@ def test_every_declared_symbol_is_exported(L):
 
 def test_packed_size_is_memory_formula_plus_header_and_padding(L):
     for N, K in ((3072, 1024), (4096, 4096), (1024, 4096), (14336, 4096), (4096, 14336), (8192, 28672)):
-        got = binding.packed_size(N, K)
-        assert got == pf.layout(N, K)["total"]
-        assert got == pf.HEADER_BYTES + pf.memory_formula_bits(N, K) // 8      # K % 1024 == 0: no padding
-    # K not a multiple of 1024 pads the code and scale regions to the next multiple
-    assert binding.packed_size(7, 1152) == 256 + 7 * 2048 // 2 + 4 * 7 * 16
+        for fmt, lay in ((1, pf.layout), (2, pf.layout_v2)):
+            got = binding.packed_size(N, K, fmt=fmt)
+            assert got == lay(N, K)["total"]
+            assert got == pf.HEADER_BYTES + pf.memory_formula_bits(N, K) // 8      # no padding at these shapes
+    # format 1: K not a multiple of 1024 pads the code and scale regions to the next multiple
+    assert binding.packed_size(7, 1152, fmt=1) == 256 + 7 * 2048 // 2 + 4 * 7 * 16
+    # format 2: an odd N stores one more row; a unit whose size is not a multiple of 16 is padded
+    assert binding.packed_size(7, 1152, fmt=2) == 256 + 4 * (1152 + 72 + 8) == pf.layout_v2(7, 1152)["total"]
+    assert binding.packed_size(3, 4224, fmt=2) == 256 + 2 * (2176 * 2 + 128 + 8 + 8) == pf.layout_v2(3, 4224)["total"]
     for bad in ((0, 128), (4, 0), (4, 100), (-1, 128)):
         assert binding.packed_size(*bad) == 0
     assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 64, 1))) == 0
-    assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 128, 2))) == 0
+    assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 128, 3))) == 0
+    assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 128, 0))) == 0
 
 
 def test_parse_header_accepts_reference_blob_and_rejects_damage(L):
     c = make_case(3, 1152, seed=2)
+    blob2 = pf.pack_reference_v2(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+    assert binding.ptqtp_parse_header(bytes(blob2[:256])) == (3, 1152, 2)
+    bad2 = blob2[:256].copy()
+    bad2[40] ^= 8         # row-pair stride no longer matches the shape
+    with pytest.raises(binding.PtqtpError):
+        binding.ptqtp_parse_header(bytes(bad2))
     blob = pf.pack_reference(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
-    assert binding.ptqtp_parse_header(bytes(blob[:256])) == (3, 1152)
+    assert binding.ptqtp_parse_header(bytes(blob[:256])) == (3, 1152, 1)
     bad = blob[:256].copy()
     bad[0] ^= 1
     with pytest.raises(binding.PtqtpError) as e:
@@ -103,6 +114,42 @@ def test_binding_refuses_cpu_tensors(L):
     with pytest.raises(TypeError):
         binding.ptqtp_gemv(torch.zeros(binding.packed_size(8, 128), dtype=torch.uint8), 8, 128,
                            torch.zeros(128, dtype=torch.float16))
+
+
+def test_reference_format2_roundtrip_layout_and_damage_detection():
+    c = make_case(5, 4224, seed=4)                       # odd N, two full slices and a 128-column tail
+    blob = pf.pack_reference_v2(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+    t1, t2, a1, a2 = pf.unpack_reference_v2(blob)
+    assert np.array_equal(t1, c["T1"]) and np.array_equal(t2, c["T2"])
+    assert np.array_equal(a1.view(np.uint16), c["alpha1"].view(np.uint16))
+    assert np.array_equal(a2.view(np.uint16), c["alpha2"].view(np.uint16))
+    # one byte by hand: row pair 1 (rows 2, 3), column 2048 + 64*3 + 16*2 + 5 = 2277:
+    # slice 1, lane block 3, sub-block 2, byte 5 -> strip offset 2176 + 16 * (2 * 32 + 3) + 5
+    strip = 2 * 2176 + 144
+    off = 256 + 1 * strip + 2176 + 16 * (2 * 32 + 3) + 5
+    want = ((int(c["T1"][2, 2277]) + 1) | (int(c["T2"][2, 2277]) + 1) << 2 | (int(c["T1"][3, 2277]) + 1) << 4
+            | (int(c["T2"][3, 2277]) + 1) << 6)
+    assert int(blob[off]) == want
+    # scale quad of row pair 0, group 17 (slice 1, second group): after the 2048 code bytes of that unit
+    q = 256 + 2176 + 2048 + 8 * 1
+    assert bytes(blob[q:q + 8]) == (c["alpha1"][0, 17].tobytes() + c["alpha2"][0, 17].tobytes()
+                                    + c["alpha1"][1, 17].tobytes() + c["alpha2"][1, 17].tobytes())
+    # the tail unit: 128 columns -> 2 lane blocks, 128 code bytes, one quad, 8 bytes of zero padding
+    tail = 256 + 2 * 2176
+    assert bytes(blob[tail + 128:tail + 136]) == (c["alpha1"][0, 32].tobytes() + c["alpha2"][0, 32].tobytes()
+                                                  + c["alpha1"][1, 32].tobytes() + c["alpha2"][1, 32].tobytes())
+    assert not blob[tail + 136:tail + 144].any()
+    # the missing row 5 is trit 0 (code 1) with zero scales
+    last = 256 + 2 * strip
+    assert (int(blob[last]) >> 4) == 0b0101
+    bad = blob.copy()
+    bad[256] |= 3
+    with pytest.raises(ValueError):
+        pf.unpack_reference_v2(bad)
+    bad = blob.copy()
+    bad[tail + 140] = 1
+    with pytest.raises(ValueError):
+        pf.unpack_reference_v2(bad)
 
 
 def test_reference_format_roundtrip_and_damage_detection():

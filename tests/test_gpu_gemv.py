@@ -10,26 +10,56 @@ from oracle.layer import layer_fp64
 from paper_2509_16989_b200 import binding
 from paper_2509_16989_b200.inputs import (LLAMA3_70B, LLAMA3_8B_UNIQUE, QWEN3_0P6B_UP, make_activations,
                                           make_case, make_weights)
-from gpu_util import assert_parity, dev, oracle_y, pack_case
+from gpu_util import FORMATS, assert_parity, dev, oracle_y, pack_case
 
 pytestmark = pytest.mark.gpu
 
 
-def run_gemv(c, **cfg):
-    packed = pack_case(c)
+def run_gemv(c, fmt=None, **cfg):
+    packed = pack_case(c, fmt)
     if cfg:
-        y = binding.ptqtp_gemv_cfg(packed, c["N"], c["K"], dev(c["x"]), **cfg)
+        y = binding.ptqtp_gemv_cfg(packed, c["N"], c["K"], dev(c["x"]), fmt=fmt, **cfg)
     else:
-        y = binding.ptqtp_gemv(packed, c["N"], c["K"], dev(c["x"]))
+        y = binding.ptqtp_gemv(packed, c["N"], c["K"], dev(c["x"]), fmt=fmt)
     torch.cuda.synchronize()
     return y.cpu().numpy()
 
 
+@pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("N,K", [(1, 128), (2, 256), (3, 1024), (5, 1152), (31, 2048), (33, 3200),
-                                 (130, 4096), (257, 5120), (64, 14336)])
-def test_small_and_ragged_shapes(N, K):
+                                 (130, 4096), (257, 5120), (64, 14336), (299, 2176), (1000, 6144),
+                                 (37, 36864)])
+def test_small_and_ragged_shapes(N, K, fmt):
     c = make_case(N, K, seed=100 + N)
-    assert_parity(run_gemv(c), oracle_y(c), c["x"], "N=%d K=%d" % (N, K))
+    assert_parity(run_gemv(c, fmt), oracle_y(c), c["x"], "fmt=%d N=%d K=%d" % (fmt, N, K))
+
+
+@pytest.mark.parametrize("warps", [1, 2, 3, 7, 8, 14, 16])
+@pytest.mark.parametrize("depth", [2, 3, 4, 6, 8])
+def test_format2_launch_configurations(warps, depth):
+    for N, K in ((67, 8192), (1000, 14336), (4, 2048)):
+        c = make_case(N, K, seed=warps * 10 + depth)
+        ref = oracle_y(c)
+        packed = pack_case(c, binding.FORMAT_V2)
+        # shared memory: x as two byte planes + block records, the slice partials, warps * depth ring slots
+        smem = (K // 64) * 136 + 2 * -(-((N + 1) // 2) // 148) * -(-K // 2048) * 4 + 16 + warps * depth * 2304
+        if smem > 227 * 1024:
+            with pytest.raises(binding.PtqtpError) as e:
+                binding.ptqtp_gemv_cfg(packed, N, K, dev(c["x"]), k_split=warps, depth=depth, fmt=binding.FORMAT_V2)
+            assert e.value.status == binding.ERR_CONFIG
+            continue
+        y = binding.ptqtp_gemv_cfg(packed, N, K, dev(c["x"]), k_split=warps, depth=depth, fmt=binding.FORMAT_V2)
+        torch.cuda.synchronize()
+        assert_parity(y.cpu().numpy(), ref, c["x"], "warps=%d depth=%d N=%d K=%d" % (warps, depth, N, K))
+
+
+def test_format2_rejects_format1_only_options():
+    c = make_case(8, 1024, seed=1)
+    packed = pack_case(c, binding.FORMAT_V2)
+    for bad in (dict(rows_per_warp=2), dict(ctas_per_sm=3), dict(arith=1), dict(k_split=17), dict(depth=5)):
+        with pytest.raises(binding.PtqtpError) as e:
+            binding.ptqtp_gemv_cfg(packed, 8, 1024, dev(c["x"]), fmt=binding.FORMAT_V2, **bad)
+        assert e.value.status == binding.ERR_CONFIG
 
 
 @pytest.mark.parametrize("R,D", [(1, 2), (1, 4), (1, 8), (2, 1), (2, 2), (2, 4), (4, 1), (4, 2)])
@@ -38,65 +68,71 @@ def test_every_launch_configuration(R, D, WS):
     for N, K in ((67, 8192), (1000, 16384)):
         c = make_case(N, K, seed=R * 10 + WS)
         ref = oracle_y(c)
-        packed = pack_case(c)
+        packed = pack_case(c, binding.FORMAT_V1)
         for arith in (0, 1, 2):
             y = binding.ptqtp_gemv_cfg(packed, N, K, dev(c["x"]), rows_per_warp=R, k_split=WS, ctas_per_sm=1,
-                                       depth=D, arith=arith)
+                                       depth=D, arith=arith, fmt=binding.FORMAT_V1)
             torch.cuda.synchronize()
             assert_parity(y.cpu().numpy(), ref, c["x"], "R=%d WS=%d D=%d arith=%d N=%d K=%d" % (R, WS, D, arith, N, K))
 
 
 def test_k_split_must_divide_the_slices():
     c = make_case(8, 3072, seed=1)
-    packed = pack_case(c)
+    packed = pack_case(c, binding.FORMAT_V1)
     with pytest.raises(binding.PtqtpError) as e:
-        binding.ptqtp_gemv_cfg(packed, 8, 3072, dev(c["x"]), rows_per_warp=1, k_split=2, depth=2)
+        binding.ptqtp_gemv_cfg(packed, 8, 3072, dev(c["x"]), rows_per_warp=1, k_split=2, depth=2,
+                               fmt=binding.FORMAT_V1)
     assert e.value.status == binding.ERR_CONFIG
 
 
 def test_unsupported_configuration_is_rejected():
     c = make_case(8, 1024, seed=1)
-    packed = pack_case(c)
+    packed = pack_case(c, binding.FORMAT_V1)
     with pytest.raises(binding.PtqtpError) as e:
-        binding.ptqtp_gemv_cfg(packed, 8, 1024, dev(c["x"]), rows_per_warp=3, k_split=1)
+        binding.ptqtp_gemv_cfg(packed, 8, 1024, dev(c["x"]), rows_per_warp=3, k_split=1, fmt=binding.FORMAT_V1)
     assert e.value.status == binding.ERR_CONFIG
 
 
-def test_config0_qwen3_up_proj():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_config0_qwen3_up_proj(fmt):
     N, K = QWEN3_0P6B_UP
     c = make_case(N, K, seed=0)
-    assert_parity(run_gemv(c), oracle_y(c), c["x"], "qwen3 up")
+    assert_parity(run_gemv(c, fmt), oracle_y(c), c["x"], "qwen3 up")
 
 
+@pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("name", sorted(LLAMA3_8B_UNIQUE))
-def test_config1_llama3_8b_shapes_full_size(name):
+def test_config1_llama3_8b_shapes_full_size(name, fmt):
     N, K = LLAMA3_8B_UNIQUE[name]
     c = make_case(N, K, seed=sorted(LLAMA3_8B_UNIQUE).index(name))
-    assert_parity(run_gemv(c), oracle_y(c), c["x"], name)
+    assert_parity(run_gemv(c, fmt), oracle_y(c), c["x"], name)
 
 
+@pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("name", sorted(LLAMA3_70B))
-def test_config3_llama3_70b_shapes_half_zero_planes(name):
+def test_config3_llama3_70b_shapes_half_zero_planes(name, fmt):
     N, K = LLAMA3_70B[name]
     c = make_case(N, K, seed=3, p_zero=0.5)
-    y = run_gemv(c)
+    y = run_gemv(c, fmt)
     rows = np.unique(np.concatenate([np.arange(0, 64), np.arange(N - 64, N),
                                      np.random.default_rng(0).integers(0, N, 1024)]))
     assert_parity(y[rows], oracle_y(c, rows), c["x"], name)
     assert np.all(np.isfinite(y))
 
 
-def test_special_planes_closed_forms():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_special_planes_closed_forms(fmt):
     N, K = 96, 2048
     c = make_case(N, K, seed=4)
+    run = lambda case: run_gemv(case, fmt)
     x64 = c["x"].astype(np.float64)
     # all-zero planes -> zero up to the fp32 rounding of (sum of x) - (sum of x)
     z = np.zeros_like(c["T1"])
     c0 = dict(c, T1=z, T2=z)
-    assert np.all(np.abs(run_gemv(c0).astype(np.float64)) <= 1e-6)
+    assert np.all(np.abs(run(c0).astype(np.float64)) <= 1e-6)
     # T1 = -T2 with equal scales -> cancels to (nearly) zero: bounded by the fp32 epilogue rounding
     cc = dict(c, T2=-c["T1"], alpha2=c["alpha1"])
-    y = run_gemv(cc).astype(np.float64)
+    y = run(cc).astype(np.float64)
     scale = np.abs(layer_fp64(c["T1"], z, c["alpha1"], c["alpha2"], c["x"]))
     assert np.all(np.abs(y) <= 2e-3 * scale.max())
     # one +1 per row, alpha1 = 1 -> gather of x (exact: a single term)
@@ -105,23 +141,25 @@ def test_special_planes_closed_forms():
     T1[np.arange(N), cols] = 1
     ones = np.ones_like(c["alpha1"])
     cg = dict(c, T1=T1, T2=z, alpha1=ones, alpha2=ones)
-    yg = run_gemv(cg).astype(np.float64)
+    yg = run(cg).astype(np.float64)
     assert np.allclose(yg, x64[cols], rtol=2e-3, atol=2e-3)
     # all +1 in plane 1 -> y_i = sum_g alpha1[i,g] * (group sums of x)
     cp = dict(c, T1=np.ones_like(c["T1"]), T2=z)
-    assert_parity(run_gemv(cp), oracle_y(cp), c["x"], "all +1")
+    assert_parity(run(cp), oracle_y(cp), c["x"], "all +1")
     cm = dict(c, T1=-np.ones_like(c["T1"]), T2=np.ones_like(c["T1"]))
-    assert_parity(run_gemv(cm), oracle_y(cm), c["x"], "all -1 / +1")
+    assert_parity(run(cm), oracle_y(cm), c["x"], "all -1 / +1")
 
 
+@pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("scale", [2.0 ** -12, 2.0 ** -6, 1.0, 2.0 ** 6, 2.0 ** 11])
-def test_activation_dynamic_range(scale):
+def test_activation_dynamic_range(scale, fmt):
     c = make_case(128, 4096, seed=6)
     c["x"] = (c["x"].astype(np.float32) * scale).astype(np.float16)
-    assert_parity(run_gemv(c), oracle_y(c), c["x"], "scale %g" % scale)
+    assert_parity(run_gemv(c, fmt), oracle_y(c), c["x"], "scale %g" % scale)
 
 
-def test_activations_with_outliers_zero_blocks_and_negative_scales():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_activations_with_outliers_zero_blocks_and_negative_scales(fmt):
     c = make_case(128, 4096, seed=7)
     x = c["x"].astype(np.float32)
     x[::97] *= 50.0                 # heavy outliers
@@ -132,31 +170,48 @@ def test_activations_with_outliers_zero_blocks_and_negative_scales():
     c["x"] = x.astype(np.float16)
     c["alpha2"] = (-c["alpha2"].astype(np.float32)).astype(np.float16)
     c["alpha1"][::3, ::2] = 0
-    assert_parity(run_gemv(c), oracle_y(c), c["x"], "outliers")
+    assert_parity(run_gemv(c, fmt), oracle_y(c), c["x"], "outliers")
 
 
-def test_output_guard_bands_and_determinism():
+def test_format2_block_fixed_point_is_exact_for_integer_activations():
+    # small integer activations and unit scales: every product and sum is an integer below 2^11,
+    # so the fp16 result must equal the exact integer sum
+    N, K = 64, 4096
+    c = make_case(N, K, seed=12)
+    rng = np.random.default_rng(3)
+    c["x"] = rng.integers(-3, 4, K).astype(np.float16)
+    c["alpha1"] = np.ones_like(c["alpha1"])
+    c["alpha2"] = np.full_like(c["alpha2"], 2.0)
+    exact = (c["T1"].astype(np.int64) @ c["x"].astype(np.int64)) + 2 * (c["T2"].astype(np.int64) @ c["x"].astype(np.int64))
+    assert np.all(np.abs(exact) < 2048)
+    y = run_gemv(c, binding.FORMAT_V2)
+    assert np.array_equal(y.astype(np.int64), exact)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_output_guard_bands_and_determinism(fmt):
     c = make_case(77, 3072, seed=8)
-    packed = pack_case(c)
+    packed = pack_case(c, fmt)
     buf = torch.full((77 + 64,), float("nan"), dtype=torch.float16, device="cuda")
     y = buf[32:32 + 77]
     # y must be 16-byte aligned: 32 halves = 64 bytes
-    binding.ptqtp_gemv(packed, 77, 3072, dev(c["x"]), y=y)
+    binding.ptqtp_gemv(packed, 77, 3072, dev(c["x"]), y=y, fmt=fmt)
     torch.cuda.synchronize()
     host = buf.cpu().numpy()
     assert np.all(np.isnan(host[:32])) and np.all(np.isnan(host[32 + 77:]))
     first = host[32:32 + 77].copy()
     for _ in range(3):
-        again = binding.ptqtp_gemv(packed, 77, 3072, dev(c["x"])).cpu().numpy()
+        again = binding.ptqtp_gemv(packed, 77, 3072, dev(c["x"]), fmt=fmt).cpu().numpy()
         assert np.array_equal(again.view(np.uint16), first.view(np.uint16))
 
 
+@pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("M", [1, 2, 3, 8, 17, 64])
-def test_gemm_skinny_matches_oracle_per_row(M):
+def test_gemm_skinny_matches_oracle_per_row(M, fmt):
     c = make_case(192, 3072, seed=20 + M, M=M)
-    packed = pack_case(c)
+    packed = pack_case(c, fmt)
     X = dev(np.atleast_2d(c["x"]))
-    Y = binding.ptqtp_gemm_skinny(packed, 192, 3072, X)
+    Y = binding.ptqtp_gemm_skinny(packed, 192, 3072, X, fmt=fmt)
     torch.cuda.synchronize()
     assert Y.shape == (M, 192)
     ref = np.atleast_2d(oracle_y(c))
@@ -173,14 +228,15 @@ def test_gemm_skinny_config2_shape_batch8_sampled_rows():
     assert_parity(Y.cpu().numpy()[:, rows], oracle_y(c, rows), c["x"], "gate_up M=8")
 
 
-def test_gemv_host_entry_point():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_gemv_host_entry_point(fmt):
     c = make_case(300, 2048, seed=9)
-    packed = pack_case(c)
+    packed = pack_case(c, fmt)
     x_host = torch.from_numpy(c["x"]).pin_memory()
     y_host = torch.empty(300, dtype=torch.float16).pin_memory()
     x_dev = torch.empty(2048, dtype=torch.float16, device="cuda")
     y_dev = torch.empty(300, dtype=torch.float16, device="cuda")
-    binding.ptqtp_gemv_host(packed, 300, 2048, x_host, y_host, x_dev, y_dev)
+    binding.ptqtp_gemv_host(packed, 300, 2048, x_host, y_host, x_dev, y_dev, fmt=fmt)
     torch.cuda.synchronize()
     assert_parity(y_host.numpy(), oracle_y(c), c["x"], "host call")
     assert np.array_equal(y_host.numpy().view(np.uint16), y_dev.cpu().numpy().view(np.uint16))

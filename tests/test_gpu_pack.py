@@ -6,14 +6,23 @@ import torch
 from oracle import packed_format as pf
 from paper_2509_16989_b200 import binding
 from paper_2509_16989_b200.inputs import LLAMA3_8B_UNIQUE, QWEN3_0P6B_UP, make_case
-from gpu_util import dev
+from gpu_util import FORMATS, dev
 
 pytestmark = pytest.mark.gpu
 
 
-def roundtrip(c):
-    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
-    T1, T2, a1, a2, st2 = binding.ptqtp_unpack(packed, c["N"], c["K"])
+def reference_blob(c, fmt):
+    writer = pf.pack_reference if fmt == binding.FORMAT_V1 else pf.pack_reference_v2
+    return writer(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+
+
+def reference_unpack(blob, fmt):
+    return (pf.unpack_reference if fmt == binding.FORMAT_V1 else pf.unpack_reference_v2)(blob)
+
+
+def roundtrip(c, fmt):
+    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=fmt)
+    T1, T2, a1, a2, st2 = binding.ptqtp_unpack(packed, c["N"], c["K"], fmt=fmt)
     torch.cuda.synchronize()
     assert int(st.item()) == 0 and int(st2.item()) == 0
     assert np.array_equal(T1.cpu().numpy(), c["T1"])
@@ -23,18 +32,23 @@ def roundtrip(c):
     return packed.cpu().numpy()
 
 
-@pytest.mark.parametrize("N,K", [(1, 128), (3, 256), (7, 1152), (33, 2048), (130, 3200), QWEN3_0P6B_UP])
-def test_roundtrip_and_bytes_match_reference_writer(N, K):
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("N,K", [(1, 128), (2, 128), (3, 256), (7, 1152), (33, 2048), (130, 3200), (9, 4224),
+                                 (64, 14336), QWEN3_0P6B_UP])
+def test_roundtrip_and_bytes_match_reference_writer(N, K, fmt):
     c = make_case(N, K, seed=N + K)
-    blob = roundtrip(c)
-    ref = pf.pack_reference(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
-    assert blob.size == ref.size == binding.packed_size(N, K)
+    blob = roundtrip(c, fmt)
+    ref = reference_blob(c, fmt)
+    assert blob.size == ref.size == binding.packed_size(N, K, fmt=fmt)
     assert np.array_equal(blob, ref)
-    t1, t2, a1, a2 = pf.unpack_reference(blob)          # the independent CPU reader agrees too
+    t1, t2, a1, a2 = reference_unpack(blob, fmt)        # the independent CPU reader agrees too
     assert np.array_equal(t1, c["T1"]) and np.array_equal(t2, c["T2"])
+    assert np.array_equal(a1.view(np.uint16), c["alpha1"].view(np.uint16))
+    assert np.array_equal(a2.view(np.uint16), c["alpha2"].view(np.uint16))
 
 
-def test_all_nine_pairs_at_every_position():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_all_nine_pairs_at_every_position(fmt):
     # row r holds pair number r at every column; then a rolling pattern so that each lane-block
     # position sees every pair next to every other pair.
     K = 2048
@@ -49,68 +63,78 @@ def test_all_nine_pairs_at_every_position():
         T2[9 + r, :] = np.array([p[1] for p in pairs], np.int8)[idx]
     c = make_case(18, K, seed=1)
     c["T1"], c["T2"] = T1, T2
-    blob = roundtrip(c)
-    assert np.array_equal(blob, pf.pack_reference(T1, T2, c["alpha1"], c["alpha2"]))
+    blob = roundtrip(c, fmt)
+    assert np.array_equal(blob, reference_blob(c, fmt))
 
 
-def test_scale_bit_patterns_are_carried_verbatim():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_scale_bit_patterns_are_carried_verbatim(fmt):
     c = make_case(4, 1024, seed=5)
     special = np.array([0x0000, 0x8000, 0x0001, 0x83FF, 0x7BFF, 0xFBFF, 0x7C00, 0xFC00, 0x7E00, 0x7C01,
                         0xFFFF, 0x3C00, 0x0400, 0x03FF, 0xBC00, 0x1234], np.uint16)
     a1 = np.resize(special, c["alpha1"].shape).astype(np.uint16)
     a2 = np.resize(special[::-1], c["alpha2"].shape).astype(np.uint16)
     c["alpha1"], c["alpha2"] = a1.view(np.float16), a2.view(np.float16)
-    roundtrip(c)
+    roundtrip(c, fmt)
 
 
+@pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("name", sorted(LLAMA3_8B_UNIQUE))
-def test_roundtrip_llama3_8b_shapes(name):
+def test_roundtrip_llama3_8b_shapes(name, fmt):
     N, K = LLAMA3_8B_UNIQUE[name]
-    roundtrip(make_case(N, K, seed=7))
+    roundtrip(make_case(N, K, seed=7), fmt)
 
 
-def test_invalid_trit_sets_device_status_and_kernel_completes():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_invalid_trit_sets_device_status_and_kernel_completes(fmt):
     c = make_case(5, 1024, seed=9)
     bad = c["T2"].copy()
     bad[3, 700] = 2
-    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(bad), dev(c["alpha1"]), dev(c["alpha2"]))
+    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(bad), dev(c["alpha1"]), dev(c["alpha2"]), fmt=fmt)
     torch.cuda.synchronize()
     assert int(st.item()) == binding.ERR_TRIT
     # the offending entry is stored as 0, everything else intact
-    T1, T2, a1, a2, st2 = binding.ptqtp_unpack(packed, 5, 1024)
+    T1, T2, a1, a2, st2 = binding.ptqtp_unpack(packed, 5, 1024, fmt=fmt)
     torch.cuda.synchronize()
     fixed = bad.copy()
     fixed[3, 700] = 0
     assert np.array_equal(T2.cpu().numpy(), fixed) and np.array_equal(T1.cpu().numpy(), c["T1"])
     bad[3, 700] = -128
-    _, st = binding.ptqtp_pack(dev(c["T1"]), dev(bad), dev(c["alpha1"]), dev(c["alpha2"]))
+    _, st = binding.ptqtp_pack(dev(c["T1"]), dev(bad), dev(c["alpha1"]), dev(c["alpha2"]), fmt=fmt)
     assert int(st.item()) == binding.ERR_TRIT
 
 
-def test_unpack_reports_header_mismatch():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_unpack_reports_header_mismatch(fmt):
     c = make_case(8, 1024, seed=10)
-    packed, _ = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
-    *_, st = binding.ptqtp_unpack(packed, 4, 2048)      # same byte size, different shape
+    packed, _ = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=fmt)
+    *_, st = binding.ptqtp_unpack(packed, 4, 2048, fmt=fmt)      # same byte size, different shape
     torch.cuda.synchronize()
     assert int(st.item()) == binding.ERR_FORMAT
+    other = binding.FORMAT_V1 + binding.FORMAT_V2 - fmt
+    if binding.packed_size(8, 1024, fmt=other) <= packed.numel():
+        *_, st = binding.ptqtp_unpack(packed, 8, 1024, fmt=other)    # a blob of the other format
+        assert int(st.item()) == binding.ERR_FORMAT
     packed[0] = 0
-    *_, st = binding.ptqtp_unpack(packed, 8, 1024)
+    *_, st = binding.ptqtp_unpack(packed, 8, 1024, fmt=fmt)
     assert int(st.item()) == binding.ERR_FORMAT
 
 
-def test_header_parses_on_host():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_header_parses_on_host(fmt):
     c = make_case(6, 1152, seed=11)
-    packed, _ = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
-    assert binding.ptqtp_parse_header(bytes(packed[:256].cpu().numpy())) == (6, 1152)
+    packed, _ = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=fmt)
+    assert binding.ptqtp_parse_header(bytes(packed[:256].cpu().numpy())) == (6, 1152, fmt)
 
 
-def test_guard_bands_untouched():
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_guard_bands_untouched(fmt):
     c = make_case(9, 1152, seed=12)
-    size = binding.packed_size(9, 1152)
+    size = binding.packed_size(9, 1152, fmt=fmt)
     buf = torch.full((size + 512,), 0xA5, dtype=torch.uint8, device="cuda")
     view = buf[256:256 + size]
-    binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), packed=view)
+    binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), packed=view, fmt=fmt)
     torch.cuda.synchronize()
     host = buf.cpu().numpy()
     assert np.all(host[:256] == 0xA5) and np.all(host[256 + size:] == 0xA5)
-    assert np.array_equal(host[256:256 + size], pf.pack_reference(c["T1"], c["T2"], c["alpha1"], c["alpha2"]))
+    assert np.array_equal(host[256:256 + size], reference_blob(c, fmt))
