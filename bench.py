@@ -424,7 +424,7 @@ def run_gpu(args):
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": "of " + peak_kind, "traffic": None,
-                     "kernel": "gemv_kernel (7 launches per step; mean over the step)",
+                     "kernel": "gemv2_kernel (7 launches per step; mean over the step)",
                      "bytes_per_launch_mean": STEP_BYTES / 7.0, "us_per_launch_mean": 1e3 * ms_per_step / 7.0},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "us_per_layer": 1e3 * e2e_ms / e2e_steps},

@@ -125,7 +125,8 @@ PTQTP_API ptqtp_status ptqtp_unpack(const ptqtp_shape *shape /* host */, const v
 /* Batch-1 decode layer y = alpha1 (.) (T1 x) + alpha2 (.) (T2 x) (Eq. 1-2 with Sec. 2.3 groups;
  * Sec. 4: additions/subtractions of x, one scale multiply per group and plane).
  * packed: device blob from ptqtp_pack (its header is not re-read; `shape` is trusted);
- * x: device fp16 [K]; y: device fp16 [N], fully overwritten.  x and y must not alias packed.
+ * x: device fp16 [K]; y: device fp16 [N], fully overwritten.  x and y must not alias packed
+ * (see also ptqtp_set_overlap).
  * Arithmetic, format 1: fp16 x times codes, fp32 accumulators, fp32 scale epilogue.
  * Arithmetic, format 2: x is turned into 16-bit block fixed point per 64 columns (exact for values within
  * 2^-5 of the block maximum, otherwise rounded to 2^-16 of it), sign-select sums are exact int32, the
@@ -155,7 +156,7 @@ PTQTP_API ptqtp_status ptqtp_gemv_host(const ptqtp_shape *shape /* host */, cons
  * arith: accumulation of the sign-selected activations -- 0 = fp32 accumulator fed by mixed-precision
  * FMAs (fp16 operands), 1 = fp16x2 chains of 4 flushed into fp32, 2 = chains of 8, -1 = library choice.
  * PTQTP_ERR_CONFIG if the combination is not built.
- * For a format-2 blob the arguments mean: rows_per_warp must be 0; k_split = warps per CTA (1..16, 0 = auto);
+ * For a format-2 blob the arguments mean: rows_per_warp must be 0; k_split = warps per CTA (1..24, 0 = auto);
  * ctas_per_sm must be 0 or 1 (one persistent CTA per SM); depth = slice units in flight per warp
  * (2, 3, 4, 6, 8; 0 = auto); arith must be -1 or 3 (integer dot products). */
 PTQTP_API ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
@@ -171,6 +172,15 @@ PTQTP_API const char *ptqtp_status_string(ptqtp_status status);
 
 /* The cudaError_t (as int) behind the calling thread's most recent PTQTP_ERR_CUDA, else 0. */
 PTQTP_API int ptqtp_last_cuda_error(void);
+
+/* Overlap of consecutive GEMV calls on one stream (process-wide switch, on by default; returns the old
+ * value).  When on, format-2 GEMV kernels are launched with programmatic stream serialization: a call may
+ * begin reading its `packed` blob while the GEMV call directly before it on the stream is still draining;
+ * x is read and y written only after all earlier work on the stream has completed, so stream order holds
+ * for them.  Consequence for the caller: the packed blob of a call must not be the output buffer of the
+ * GEMV call directly before it.  Work of any other kind before a call is always complete before the call
+ * reads anything.  Works inside CUDA graph capture. */
+PTQTP_API int ptqtp_set_overlap(int enabled);
 
 /* Library version: major*10000 + minor*100 + patch. */
 PTQTP_API int ptqtp_version(void);

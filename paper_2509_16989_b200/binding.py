@@ -23,7 +23,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_SIZE, ERR_TRIT, ERR_FORMAT, ERR_CUDA, ER
 
 EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny",
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
-           "ptqtp_last_cuda_error", "ptqtp_version")
+           "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap")
 
 
 class PtqtpError(RuntimeError):
@@ -71,6 +71,8 @@ def lib():
         L.ptqtp_status_string.argtypes = [ctypes.c_int]
         L.ptqtp_last_cuda_error.restype = ctypes.c_int
         L.ptqtp_version.restype = ctypes.c_int
+        L.ptqtp_set_overlap.restype = ctypes.c_int
+        L.ptqtp_set_overlap.argtypes = [ctypes.c_int]
         _lib = L
     return _lib
 
@@ -192,6 +194,11 @@ def ptqtp_gemv_host(packed, N, K, x_host, y_host, x_dev, y_dev, stream=None, fmt
                                _stream_ptr(stream))
     _check(st, "ptqtp_gemv_host")
     return y_host
+
+
+def ptqtp_set_overlap(enabled):
+    """Switch the overlap of consecutive GEMV calls (programmatic dependent launch); returns the old setting."""
+    return bool(lib().ptqtp_set_overlap(1 if enabled else 0))
 
 
 def ptqtp_parse_header(header_bytes):

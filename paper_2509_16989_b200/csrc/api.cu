@@ -5,6 +5,9 @@
 namespace ptqtp {
 
 static thread_local int g_last_cuda_error = 0;
+static int g_overlap = 1;
+
+bool overlap_enabled() { return g_overlap != 0; }
 
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
 
@@ -190,6 +193,12 @@ const char* ptqtp_status_string(ptqtp_status status) {
 }
 
 int ptqtp_last_cuda_error(void) { return g_last_cuda_error; }
+
+int ptqtp_set_overlap(int enabled) {
+    const int old = g_overlap;
+    g_overlap = enabled ? 1 : 0;
+    return old;
+}
 
 int ptqtp_version(void) { return 100; }
 

@@ -29,6 +29,8 @@ namespace ptqtp {
 namespace {
 
 constexpr int kSlot = 2048 + 256;          // ring slot: 128 atoms of 16 B + one 8-byte scale quad per lane
+constexpr int kMaxWarps2 = 24;
+constexpr int kMaxThreads2 = kMaxWarps2 * 32;
 
 __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
     const unsigned d = (unsigned)__cvta_generic_to_shared(dst_smem);
@@ -54,70 +56,65 @@ __device__ __forceinline__ int dot_uu(uint32_t a, uint32_t x, int c) {
     return d;
 }
 
-// Convert x to block fixed point in shared memory.
+// Convert 8 activations (one uint4 of fp16) to block fixed point and store them in shared memory.
 //   xhi, xlo : [K/64 blocks][16 words]  bytes of hi_j / lo_j in column order
-//   meta     : [K/64 blocks] (2^-s as float, sum_j X_j as int)
-// Eight adjacent threads share a 64-column block (8 columns each).
-__device__ __forceinline__ void stage_x(int K, const __half* __restrict__ x, uint32_t* xhi, uint32_t* xlo,
-                                        int2* meta) {
-    const int threads = blockDim.x;
-    for (int wbase = (threadIdx.x & ~31) * 8; wbase < K; wbase += threads * 8) {     // warp-uniform loop
-        const int base = wbase + (threadIdx.x & 31) * 8;
-        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-        if (base < K) raw = __ldg(reinterpret_cast<const uint4*>(x + base));
-        const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-        float f[8];
-        float mx = 0.f;
+//   meta     : [K/64 blocks] (2^-s as float bits, sum_j X_j)
+// Eight adjacent threads share a 64-column block (8 columns each); the whole warp must call this.
+__device__ __forceinline__ void convert_x8(uint4 raw, int base, bool valid, uint32_t* xhi, uint32_t* xlo, int2* meta) {
+    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+    float f[8];
+    float mx = 0.f;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float2 v = __half22float2(h2[e]);
-            f[2 * e] = v.x;
-            f[2 * e + 1] = v.y;
-            mx = fmaxf(mx, fmaxf(fabsf(v.x), fabsf(v.y)));
+    for (int e = 0; e < 4; ++e) {
+        const float2 v = __half22float2(h2[e]);
+        f[2 * e] = v.x;
+        f[2 * e + 1] = v.y;
+        mx = fmaxf(mx, fmaxf(fabsf(v.x), fabsf(v.y)));
+    }
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    // exponent of the block maximum: fp16 inputs keep it within [-24, 15]
+    int s = 0;
+    if (mx > 0.f) {
+        int ex = (int)((__float_as_uint(mx) >> 23) & 0xffu) - 127;
+        ex = min(max(ex, -24), 15);
+        s = 14 - ex;
+    }
+    const float scale = __uint_as_float((uint32_t)(127 + s) << 23);
+    int X[8];
+    int sum = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        X[e] = __float2int_rn(f[e] * scale);
+        X[e] = min(max(X[e], -32767), 32767);
+        sum += X[e];
+    }
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    uint32_t hw[2], lw[2];
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+        hw[w] = 0u;
+        lw[w] = 0u;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int v = X[4 * w + b];
+            hw[w] |= (uint32_t)((v >> 8) & 0xff) << (8 * b);
+            lw[w] |= (uint32_t)(v & 0xff) << (8 * b);
         }
-#pragma unroll
-        for (int o = 1; o < 8; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        // exponent of the block maximum: fp16 inputs keep it within [-24, 15]
-        int s = 0;
-        if (mx > 0.f) {
-            int ex = (int)((__float_as_uint(mx) >> 23) & 0xffu) - 127;
-            ex = min(max(ex, -24), 15);
-            s = 14 - ex;
-        }
-        const float scale = __uint_as_float((uint32_t)(127 + s) << 23);
-        int X[8];
-        int sum = 0;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            X[e] = __float2int_rn(f[e] * scale);
-            X[e] = min(max(X[e], -32767), 32767);
-            sum += X[e];
-        }
-#pragma unroll
-        for (int o = 1; o < 8; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        uint32_t hw[2], lw[2];
-#pragma unroll
-        for (int w = 0; w < 2; ++w) {
-            hw[w] = 0u;
-            lw[w] = 0u;
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const int v = X[4 * w + b];
-                hw[w] |= (uint32_t)((v >> 8) & 0xff) << (8 * b);
-                lw[w] |= (uint32_t)(v & 0xff) << (8 * b);
-            }
-        }
-        if (base < K) {
-            const int blk = base >> 6, tt = (base >> 3) & 7;
-            *reinterpret_cast<uint2*>(xhi + blk * 16 + 2 * tt) = make_uint2(hw[0], hw[1]);
-            *reinterpret_cast<uint2*>(xlo + blk * 16 + 2 * tt) = make_uint2(lw[0], lw[1]);
-            if (tt == 0) meta[blk] = make_int2((int)((uint32_t)(127 - s) << 23), sum);
-        }
+    }
+    if (valid) {
+        const int blk = base >> 6, tt = (base >> 3) & 7;
+        *reinterpret_cast<uint2*>(xhi + blk * 16 + 2 * tt) = make_uint2(hw[0], hw[1]);
+        *reinterpret_cast<uint2*>(xlo + blk * 16 + 2 * tt) = make_uint2(lw[0], lw[1]);
+        if (tt == 0) meta[blk] = make_int2((int)((uint32_t)(127 - s) << 23), sum);
     }
 }
 
+constexpr int kPre = 4;                    // x loads per thread issued ahead of the weight stream
+
 template <int D>
-__global__ void __launch_bounds__(512, 1)
+__global__ void __launch_bounds__(kMaxThreads2, 1)
 gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
              __half* __restrict__ y, int rows_cap) {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -129,7 +126,10 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     const int warps = blockDim.x >> 5;
     const size_t ring_off = ((size_t)nblk * 136 + (size_t)rows_cap * L.slices * 4 + 15) / 16 * 16;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned char* ring = smem + ring_off + (size_t)warp * D * kSlot;
+    unsigned char* ring_lane = smem + ring_off + (size_t)warp * D * kSlot + lane * 16;
+
+    // Let the next kernel on the stream start its own weight prefetch while this one drains.
+    asm volatile("griddepcontrol.launch_dependents;");
 
     // this CTA's row pairs, and this warp's share of their slice units
     const int rp0 = (int)((long long)blockIdx.x * L.nrp / gridDim.x);
@@ -141,99 +141,134 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     const bool idle = wi >= m;
     const int n_sl = idle ? 0 : (S - sl_lane + Wc - 1) / Wc;
     const int n_rp = idle ? 0 : max(0, (rp1 - rp0 - wi + m - 1) / m);
-    const int total = n_sl * n_rp;
-    const unsigned char* codes = packed + L.codes_off;
+    const unsigned char* codes = packed + L.codes_off + (size_t)(rp0 + wi) * L.strip;
+    const size_t rp_stride = (size_t)m * L.strip;
 
-    // prefetch cursor
-    int pt = 0, pj = 0, pq = 0;
-    auto issue = [&](int slot) {
-        if (pq < total) {
-            const int sl = sl_lane + pt * Wc, rp = rp0 + wi + pj * m;
-            const int active = sl == S - 1 ? L.last_active : 32;
-            const unsigned char* src = codes + (size_t)rp * L.strip + (size_t)sl * kUnit2;
-            unsigned char* dst = ring + slot * kSlot;
-            if (lane < active) {
+    // prefetch cursor: slice pass pt, row pair pj, source of the next unit, ring slot offset
+    int pt = n_rp > 0 ? 0 : n_sl, pj = 0, pslot = 0;
+    int pactive = sl_lane == S - 1 ? L.last_active : 32;
+    const unsigned char* psrc = codes + (size_t)sl_lane * kUnit2;
+    auto issue = [&]() {
+        if (pt < n_sl) {
+            if (lane < pactive) {
+                const unsigned char* src = psrc + lane * 16;
+                unsigned char* dst = ring_lane + pslot;
+                const int istride = pactive * 16;
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    cp_async16(dst + (i * 32 + lane) * 16, src + ((size_t)i * active + lane) * 16);
-                cp_async8(dst + 2048 + lane * 8, src + (size_t)active * 64 + (lane >> 1) * 8);
+                for (int i = 0; i < 4; ++i) cp_async16(dst + i * 512, src + i * istride);
+                cp_async8(dst + 2048 - lane * 8, psrc + pactive * 64 + (lane >> 1) * 8);
             }
-            ++pq;
-            if (++pj == n_rp) { pj = 0; ++pt; }
+            psrc += rp_stride;
+            if (++pj == n_rp) {
+                pj = 0;
+                ++pt;
+                const int sl = sl_lane + pt * Wc;
+                pactive = sl == S - 1 ? L.last_active : 32;
+                psrc = codes + (size_t)sl * kUnit2;
+            }
         }
         cp_async_commit();
+        pslot = pslot + kSlot == D * kSlot ? 0 : pslot + kSlot;
     };
+    // One unit per warp goes out before anything else: the packed planes do not depend on earlier work of the
+    // stream (see ptqtp_gemv), x and y do.  Then wait for that earlier work, fetch x ahead of the rest of
+    // the weight stream (the whole CTA waits for x; its loads must not queue behind the stream), then fill
+    // the ring.
+    issue();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int xstep = blockDim.x * 8;
+    const int xbase = (threadIdx.x & ~31) * 8, xlane = (threadIdx.x & 31) * 8;
+    uint4 xraw[kPre];
 #pragma unroll
-    for (int d = 0; d < D; ++d) issue(d);
+    for (int p = 0; p < kPre; ++p) {
+        const int base = xbase + p * xstep + xlane;
+        xraw[p] = make_uint4(0u, 0u, 0u, 0u);
+        if (base < L.k) xraw[p] = __ldg(reinterpret_cast<const uint4*>(x + base));
+    }
+#pragma unroll
+    for (int d = 1; d < D; ++d) issue();
 
-    stage_x(L.k, x, xhi, xlo, meta);
+#pragma unroll
+    for (int p = 0; p < kPre; ++p) {
+        if (xbase + p * xstep < L.k) {
+            const int base = xbase + p * xstep + xlane;
+            convert_x8(xraw[p], base, base < L.k, xhi, xlo, meta);
+        }
+    }
+    for (int wb = xbase + kPre * xstep; wb < L.k; wb += xstep) {       // very long K: the rest, loaded late
+        const int base = wb + xlane;
+        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+        if (base < L.k) raw = __ldg(reinterpret_cast<const uint4*>(x + base));
+        convert_x8(raw, base, base < L.k, xhi, xlo, meta);
+    }
     __syncthreads();
 
-    uint32_t xh[16], xl[16];
-    float c = 0.f;
-    int neg[4] = {0, 0, 0, 0};
-    int ct = 0, cj = 0;
-    bool live = false;
-    for (int q = 0; q < total; ++q) {
-        const int slot = q % D;
-        const int sl = sl_lane + ct * Wc, rp = rp0 + wi + cj * m;
-        if (cj == 0) {                                  // new slice: load this lane's X block
-            const int active = sl == S - 1 ? L.last_active : 32;
-            live = lane < active;
-            const int blk = sl * 32 + (live ? lane : 0);
+    int cslot = 0;
+    for (int t = 0; t < n_sl; ++t) {
+        const int sl = sl_lane + t * Wc;
+        const int active = sl == S - 1 ? L.last_active : 32;
+        const bool live = lane < active;
+        // this lane's X block for the slice stays in registers
+        uint32_t xh[16], xl[16];
+        const int blk = sl * 32 + (live ? lane : 0);
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                const uint4 a = *reinterpret_cast<const uint4*>(xhi + blk * 16 + 4 * v);
-                const uint4 b = *reinterpret_cast<const uint4*>(xlo + blk * 16 + 4 * v);
-                xh[4 * v] = a.x; xh[4 * v + 1] = a.y; xh[4 * v + 2] = a.z; xh[4 * v + 3] = a.w;
-                xl[4 * v] = b.x; xl[4 * v + 1] = b.y; xl[4 * v + 2] = b.z; xl[4 * v + 3] = b.w;
-            }
-            const int2 mt = meta[blk];
-            c = __int_as_float(mt.x);
-#pragma unroll
-            for (int f = 0; f < 4; ++f) neg[f] = -(mt.y << (2 * f));
+        for (int v = 0; v < 4; ++v) {
+            const uint4 a = *reinterpret_cast<const uint4*>(xhi + blk * 16 + 4 * v);
+            const uint4 b = *reinterpret_cast<const uint4*>(xlo + blk * 16 + 4 * v);
+            xh[4 * v] = a.x; xh[4 * v + 1] = a.y; xh[4 * v + 2] = a.z; xh[4 * v + 3] = a.w;
+            xl[4 * v] = b.x; xl[4 * v + 1] = b.y; xl[4 * v + 2] = b.z; xl[4 * v + 3] = b.w;
         }
-        cp_async_wait<D - 1>();
-        const unsigned char* buf = ring + slot * kSlot;
-        float y0 = 0.f, y1 = 0.f;
-        if (live) {
+        const int2 mt = meta[blk];
+        const float c0 = live ? __int_as_float(mt.x) : 0.f, c1 = 0.0625f * c0;
+        const int xsum = mt.y;
+        float* ppart = partial + (size_t)wi * 2 * S + sl + (lane >> 4) * S;
+        for (int j = 0; j < n_rp; ++j) {
+            cp_async_wait<D - 1>();
+            const unsigned char* buf = ring_lane + cslot;
+            // Fields 0..2 are masked out of each code word; the unmasked word gives the sum of all four fields
+            // (a byte is q0 + 4 q1 + 16 q2 + 64 q3 <= 170), so field 3 is "all" minus the other three.
             int ah[4] = {0, 0, 0, 0};
-            int al[4] = {neg[0], neg[1], neg[2], neg[3]};
+            int al[4] = {0, 0, 0, 0};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint4 cw = *reinterpret_cast<const uint4*>(buf + (i * 32 + lane) * 16);
+                const uint4 cw = *reinterpret_cast<const uint4*>(buf + i * 512);
                 const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
                 for (int ww = 0; ww < 4; ++ww) {
 #pragma unroll
-                    for (int f = 0; f < 4; ++f) {
+                    for (int f = 0; f < 3; ++f) {
                         const uint32_t mk = w[ww] & (0x03030303u << (2 * f));
                         ah[f] = dot_us(mk, xh[4 * i + ww], ah[f]);
                         al[f] = dot_uu(mk, xl[4 * i + ww], al[f]);
                     }
+                    ah[3] = dot_us(w[ww], xh[4 * i + ww], ah[3]);
+                    al[3] = dot_uu(w[ww], xl[4 * i + ww], al[3]);
                 }
             }
-            const uint2 sc = *reinterpret_cast<const uint2*>(buf + 2048 + lane * 8);
+            const uint2 sc = *reinterpret_cast<const uint2*>(buf + 2048 - lane * 8);
             const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));   // alpha1, alpha2 of row 0
             const float2 s1 = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));   // ... of row 1
+            // Q[f] = 4^f * sum_j q_j X_j per field; subtracting 4^f * sum_j X_j turns codes into trits
+            int Q[4];
+#pragma unroll
+            for (int f = 0; f < 4; ++f) Q[f] = (ah[f] << 8) + al[f];
+            Q[3] -= Q[0] + Q[1] + Q[2];
             float F[4];
 #pragma unroll
-            for (int f = 0; f < 4; ++f) F[f] = (float)((ah[f] << 8) + al[f]);              // 4^f * sum_j t_j X_j
-            y0 = c * fmaf(s0.x, F[0], 0.25f * (s0.y * F[1]));
-            y1 = (0.0625f * c) * fmaf(s1.x, F[2], 0.25f * (s1.y * F[3]));
-        }
-        issue(slot);
+            for (int f = 0; f < 4; ++f) F[f] = (float)(Q[f] - (xsum << (2 * f)));
+            // lanes past the slice's columns hold stale ring bytes and are zeroed explicitly
+            float y0 = live ? c0 * fmaf(s0.x, F[0], 0.25f * (s0.y * F[1])) : 0.f;
+            float y1 = live ? c1 * fmaf(s1.x, F[2], 0.25f * (s1.y * F[3])) : 0.f;
+            issue();
+            cslot = cslot + kSlot == D * kSlot ? 0 : cslot + kSlot;
+            // lanes 0-15 reduce row 0, lanes 16-31 row 1
+            const float send = (lane & 16) ? y0 : y1;
+            float v = ((lane & 16) ? y1 : y0) + __shfl_xor_sync(0xffffffffu, send, 16);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            y0 += __shfl_xor_sync(0xffffffffu, y0, o);
-            y1 += __shfl_xor_sync(0xffffffffu, y1, o);
+            for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if ((lane & 15) == 0) *ppart = v;
+            ppart += (size_t)m * 2 * S;
         }
-        if (lane == 0) {
-            float* p = partial + (size_t)(rp - rp0) * 2 * S + sl;
-            p[0] = y0;
-            p[S] = y1;
-        }
-        if (++cj == n_rp) { cj = 0; ++ct; }
     }
     cp_async_wait<0>();
     __syncthreads();
@@ -264,9 +299,20 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
         if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
         configured[dev] = smem;
     }
-    kern<<<grid, warps * 32, smem, st>>>(L, static_cast<const unsigned char*>(packed),
-                                         reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap);
-    return check_launch();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(warps * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_enabled() ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, L, static_cast<const unsigned char*>(packed),
+                                       reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap);
+    if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
+    return PTQTP_OK;
 }
 
 }  // namespace
@@ -274,16 +320,20 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps, int depth,
                           cudaStream_t st) {
     const int S = L.slices;
-    if (warps == 0) {
-        // the multiple of the slice count closest below 16 warps, so every slice lane has as many warps
-        warps = S <= 16 ? S * (16 / S) : 16;
-    }
-    if (warps < 1 || warps > 16) return PTQTP_ERR_CONFIG;
     const int grid = min(sm_count(), L.nrp);
+    if (warps == 0) {
+        // A multiple of the slice count (every slice lane gets as many warps): about 12 warps when a CTA has
+        // many slice units to stream, about 8 when it has few (measured on the LLaMA-3 shapes).
+        const long units_per_cta = (long)((L.nrp + grid - 1) / grid) * S;
+        const int target = units_per_cta >= 64 ? 12 : 8;
+        warps = S >= kMaxWarps2 ? kMaxWarps2 : S * max(1, (target + S / 2) / S);
+        if (warps > kMaxWarps2) warps = S * (kMaxWarps2 / S);
+    }
+    if (warps < 1 || warps > kMaxWarps2) return PTQTP_ERR_CONFIG;
     const int rows_cap = 2 * ((L.nrp + grid - 1) / grid);
     const size_t budget = 227 * 1024;
     if (depth == 0) {
-        depth = 4;
+        depth = 3;
         while (depth > 2 && smem_bytes(L, rows_cap, warps, depth) > budget) --depth;
     }
     const size_t smem = smem_bytes(L, rows_cap, warps, depth);

@@ -100,5 +100,6 @@ ptqtp_status launch_unpack2(const Layout2& L, const void* packed, int8_t* T1, in
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
                           int depth, cudaStream_t st);
 int sm_count();
+bool overlap_enabled();           // programmatic dependent launch of the GEMV kernels (ptqtp_set_overlap)
 
 }  // namespace ptqtp

@@ -34,7 +34,7 @@ def test_small_and_ragged_shapes(N, K, fmt):
     assert_parity(run_gemv(c, fmt), oracle_y(c), c["x"], "fmt=%d N=%d K=%d" % (fmt, N, K))
 
 
-@pytest.mark.parametrize("warps", [1, 2, 3, 7, 8, 14, 16])
+@pytest.mark.parametrize("warps", [1, 2, 3, 7, 8, 14, 16, 21, 24])
 @pytest.mark.parametrize("depth", [2, 3, 4, 6, 8])
 def test_format2_launch_configurations(warps, depth):
     for N, K in ((67, 8192), (1000, 14336), (4, 2048)):
@@ -56,7 +56,7 @@ def test_format2_launch_configurations(warps, depth):
 def test_format2_rejects_format1_only_options():
     c = make_case(8, 1024, seed=1)
     packed = pack_case(c, binding.FORMAT_V2)
-    for bad in (dict(rows_per_warp=2), dict(ctas_per_sm=3), dict(arith=1), dict(k_split=17), dict(depth=5)):
+    for bad in (dict(rows_per_warp=2), dict(ctas_per_sm=3), dict(arith=1), dict(k_split=25), dict(depth=5)):
         with pytest.raises(binding.PtqtpError) as e:
             binding.ptqtp_gemv_cfg(packed, 8, 1024, dev(c["x"]), fmt=binding.FORMAT_V2, **bad)
         assert e.value.status == binding.ERR_CONFIG
@@ -260,3 +260,55 @@ def test_decomposed_weights_end_to_end():
     dense = W.astype(np.float64) @ c["x"].astype(np.float64)
     rel = np.linalg.norm(y.astype(np.float64) - dense) / np.linalg.norm(dense)
     assert rel < 2.5 * err
+
+
+@pytest.mark.parametrize("graph", [False, True])
+def test_overlapped_chain_keeps_stream_order(graph):
+    # y1 = layer1(x), y2 = layer2(y1), y3 = layer1(y2): each call's x is the previous call's y, so a call
+    # that read x before its predecessor finished would be caught.  Checked link by link against the oracle.
+    N = K = 2048
+    c1, c2 = make_case(N, K, seed=50), make_case(N, K, seed=51)
+    c1["alpha1"] = (c1["alpha1"].astype(np.float32) * 1.5).astype(np.float16)      # keep the chain's magnitude near 1
+    c2["alpha1"] = (c2["alpha1"].astype(np.float32) * 1.5).astype(np.float16)
+    p1, p2 = pack_case(c1, binding.FORMAT_V2), pack_case(c2, binding.FORMAT_V2)
+    x = dev(c1["x"])
+    ys = [torch.empty(N, dtype=torch.float16, device="cuda") for _ in range(3)]
+    assert binding.ptqtp_set_overlap(True) in (True, False)
+
+    def chain():
+        binding.ptqtp_gemv(p1, N, K, x, y=ys[0], fmt=binding.FORMAT_V2)
+        binding.ptqtp_gemv(p2, N, K, ys[0], y=ys[1], fmt=binding.FORMAT_V2)
+        binding.ptqtp_gemv(p1, N, K, ys[1], y=ys[2], fmt=binding.FORMAT_V2)
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        chain()
+        stream.synchronize()
+        if graph:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for _ in range(8):
+                    chain()
+        for y in ys:
+            y.zero_()
+        for _ in range(5):
+            if graph:
+                g.replay()
+            else:
+                for _ in range(8):
+                    chain()
+        stream.synchronize()
+    h = [y.cpu().numpy() for y in ys]
+    for cc, xin, yout, what in ((c1, c1["x"], h[0], "link 1"), (c2, h[0], h[1], "link 2"), (c1, h[1], h[2], "link 3")):
+        ref = oracle_y(dict(cc, x=xin))
+        assert_parity(yout, ref, xin, what)
+    # and with the overlap switched off the results are bit-identical
+    assert binding.ptqtp_set_overlap(False) is True
+    try:
+        with torch.cuda.stream(stream):
+            chain()
+            stream.synchronize()
+        for y, ref in zip(ys, h):
+            assert np.array_equal(y.cpu().numpy().view(np.uint16), ref.view(np.uint16))
+    finally:
+        binding.ptqtp_set_overlap(True)
