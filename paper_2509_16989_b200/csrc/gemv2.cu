@@ -62,46 +62,46 @@ __device__ __forceinline__ int dot_uu(uint32_t a, uint32_t x, int c) {
 // Eight adjacent threads share a 64-column block (8 columns each); the whole warp must call this.
 __device__ __forceinline__ void convert_x8(uint4 raw, int base, bool valid, uint32_t* xhi, uint32_t* xlo, int2* meta) {
     const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-    float f[8];
-    float mx = 0.f;
+    // block maximum of |x| on the fp16 bit patterns (ordered like the values once the sign is cleared)
+    const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+    uint32_t mxb = 0u;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const float2 v = __half22float2(h2[e]);
-        f[2 * e] = v.x;
-        f[2 * e + 1] = v.y;
-        mx = fmaxf(mx, fmaxf(fabsf(v.x), fabsf(v.y)));
+        const uint32_t a = rw[e] & 0x7fff7fffu;
+        mxb = max(mxb, max(a & 0xffffu, a >> 16));
     }
 #pragma unroll
-    for (int o = 1; o < 8; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    // exponent of the block maximum: fp16 inputs keep it within [-24, 15]
+    for (int o = 1; o < 8; o <<= 1) mxb = max(mxb, __shfl_xor_sync(0xffffffffu, mxb, o));
+    // exponent of the block maximum, in [-24, 15] for finite inputs; subnormal fp16 (exponent field 0) are
+    // integers times 2^-24
     int s = 0;
-    if (mx > 0.f) {
-        int ex = (int)((__float_as_uint(mx) >> 23) & 0xffu) - 127;
-        ex = min(max(ex, -24), 15);
+    if (mxb != 0u) {
+        const int ef = (int)(mxb >> 10);
+        const int ex = ef ? ef - 15 : (31 - __clz((int)mxb)) - 24;
         s = 14 - ex;
     }
     const float scale = __uint_as_float((uint32_t)(127 + s) << 23);
     int X[8];
     int sum = 0;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        X[e] = __float2int_rn(f[e] * scale);
-        X[e] = min(max(X[e], -32767), 32767);
-        sum += X[e];
+    for (int e = 0; e < 4; ++e) {
+        const float2 v = __half22float2(h2[e]);
+        // x * 2^s is exact and below 2^15 in magnitude; adding 1.5 * 2^23 rounds it to the nearest integer
+        // (ties to even) and leaves that integer in the low mantissa bits
+        X[2 * e] = __float_as_int(fmaf(v.x, scale, 12582912.f)) - 0x4B400000;
+        X[2 * e + 1] = __float_as_int(fmaf(v.y, scale, 12582912.f)) - 0x4B400000;
+        sum += X[2 * e] + X[2 * e + 1];
     }
 #pragma unroll
     for (int o = 1; o < 8; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     uint32_t hw[2], lw[2];
 #pragma unroll
     for (int w = 0; w < 2; ++w) {
-        hw[w] = 0u;
-        lw[w] = 0u;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const int v = X[4 * w + b];
-            hw[w] |= (uint32_t)((v >> 8) & 0xff) << (8 * b);
-            lw[w] |= (uint32_t)(v & 0xff) << (8 * b);
-        }
+        // byte 0 (lo) and byte 1 (hi) of four consecutive X gathered into one word each
+        const uint32_t lo01 = __byte_perm(X[4 * w], X[4 * w + 1], 0x0040), lo23 = __byte_perm(X[4 * w + 2], X[4 * w + 3], 0x0040);
+        const uint32_t hi01 = __byte_perm(X[4 * w], X[4 * w + 1], 0x0051), hi23 = __byte_perm(X[4 * w + 2], X[4 * w + 3], 0x0051);
+        lw[w] = __byte_perm(lo01, lo23, 0x5410);
+        hw[w] = __byte_perm(hi01, hi23, 0x5410);
     }
     if (valid) {
         const int blk = base >> 6, tt = (base >> 3) & 7;
@@ -220,7 +220,9 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
         }
         const int2 mt = meta[blk];
         const float c0 = live ? __int_as_float(mt.x) : 0.f, c1 = 0.0625f * c0;
-        const int xsum = mt.y;
+        // sum_j t_j X_j = sum_j q_j X_j - sum_j X_j: the low accumulators start at minus 4^f times the block sum;
+        // the unmasked word stands for all four fields at once and starts at minus (1 + 4 + 16 + 64) times it
+        const int n0 = -mt.y, n1 = -(mt.y << 2), n2 = -(mt.y << 4), n3 = -(mt.y * 85);
         float* ppart = partial + (size_t)wi * 2 * S + sl + (lane >> 4) * S;
         for (int j = 0; j < n_rp; ++j) {
             cp_async_wait<D - 1>();
@@ -228,7 +230,7 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
             // Fields 0..2 are masked out of each code word; the unmasked word gives the sum of all four fields
             // (a byte is q0 + 4 q1 + 16 q2 + 64 q3 <= 170), so field 3 is "all" minus the other three.
             int ah[4] = {0, 0, 0, 0};
-            int al[4] = {0, 0, 0, 0};
+            int al[4] = {n0, n1, n2, n3};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint4 cw = *reinterpret_cast<const uint4*>(buf + i * 512);
@@ -248,17 +250,12 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
             const uint2 sc = *reinterpret_cast<const uint2*>(buf + 2048 - lane * 8);
             const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));   // alpha1, alpha2 of row 0
             const float2 s1 = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));   // ... of row 1
-            // Q[f] = 4^f * sum_j q_j X_j per field; subtracting 4^f * sum_j X_j turns codes into trits
-            int Q[4];
-#pragma unroll
-            for (int f = 0; f < 4; ++f) Q[f] = (ah[f] << 8) + al[f];
-            Q[3] -= Q[0] + Q[1] + Q[2];
-            float F[4];
-#pragma unroll
-            for (int f = 0; f < 4; ++f) F[f] = (float)(Q[f] - (xsum << (2 * f)));
+            // Q0..Q2 = 4^f * sum_j t_j X_j of fields 0..2; the unmasked word minus those three is field 3's
+            const int Q0 = (ah[0] << 8) + al[0], Q1 = (ah[1] << 8) + al[1], Q2 = (ah[2] << 8) + al[2];
+            const int Q3 = (ah[3] << 8) + al[3] - Q0 - Q1 - Q2;
             // lanes past the slice's columns hold stale ring bytes and are zeroed explicitly
-            float y0 = live ? c0 * fmaf(s0.x, F[0], 0.25f * (s0.y * F[1])) : 0.f;
-            float y1 = live ? c1 * fmaf(s1.x, F[2], 0.25f * (s1.y * F[3])) : 0.f;
+            float y0 = live ? c0 * fmaf(0.25f, s0.y * (float)Q1, s0.x * (float)Q0) : 0.f;
+            float y1 = live ? c1 * fmaf(0.25f, s1.y * (float)Q3, s1.x * (float)Q2) : 0.f;
             issue();
             cslot = cslot + kSlot == D * kSlot ? 0 : cslot + kSlot;
             // lanes 0-15 reduce row 0, lanes 16-31 row 1
