@@ -156,7 +156,7 @@ PTQTP_API ptqtp_status ptqtp_gemv_host(const ptqtp_shape *shape /* host */, cons
  * arith: accumulation of the sign-selected activations -- 0 = fp32 accumulator fed by mixed-precision
  * FMAs (fp16 operands), 1 = fp16x2 chains of 4 flushed into fp32, 2 = chains of 8, -1 = library choice.
  * PTQTP_ERR_CONFIG if the combination is not built.
- * For a format-2 blob the arguments mean: rows_per_warp must be 0; k_split = warps per CTA (1..24, 0 = auto);
+ * For a format-2 blob the arguments mean: rows_per_warp must be 0; k_split = warps per CTA (1..16, 0 = auto);
  * ctas_per_sm must be 0 or 1 (one persistent CTA per SM); depth = slice units in flight per warp
  * (2, 3, 4, 6, 8; 0 = auto); arith must be -1 or 3 (integer dot products). */
 PTQTP_API ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,

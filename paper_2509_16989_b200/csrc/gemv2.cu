@@ -29,7 +29,7 @@ namespace ptqtp {
 namespace {
 
 constexpr int kSlot = 2048 + 256;          // ring slot: 128 atoms of 16 B + one 8-byte scale quad per lane
-constexpr int kMaxWarps2 = 24;
+constexpr int kMaxWarps2 = 16;
 constexpr int kMaxThreads2 = kMaxWarps2 * 32;
 
 __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
@@ -319,10 +319,10 @@ ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* 
     const int S = L.slices;
     const int grid = min(sm_count(), L.nrp);
     if (warps == 0) {
-        // A multiple of the slice count (every slice lane gets as many warps): about 12 warps when a CTA has
+        // A multiple of the slice count (every slice lane gets as many warps): about 16 warps when a CTA has
         // many slice units to stream, about 8 when it has few (measured on the LLaMA-3 shapes).
         const long units_per_cta = (long)((L.nrp + grid - 1) / grid) * S;
-        const int target = units_per_cta >= 64 ? 12 : 8;
+        const int target = units_per_cta >= 64 ? 16 : 8;
         warps = S >= kMaxWarps2 ? kMaxWarps2 : S * max(1, (target + S / 2) / S);
         if (warps > kMaxWarps2) warps = S * (kMaxWarps2 / S);
     }
