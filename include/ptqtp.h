@@ -136,7 +136,11 @@ PTQTP_API ptqtp_status ptqtp_gemv(const ptqtp_shape *shape /* host */, const voi
                         const uint16_t *x, uint16_t *y, void *stream);
 
 /* Small-batch variant: Y[m,:] = layer(X[m,:]) for m < M, 1 <= M <= PTQTP_MAX_BATCH.
- * X: device fp16 [M*K] row-major; Y: device fp16 [M*N] row-major.  Same definition per row of X. */
+ * X: device fp16 [M*K] row-major; Y: device fp16 [M*N] row-major.  Same definition per row of X.
+ * Format 2, M >= 2: the planes are decoded once per pass of up to 8 batch rows (fewer when K is long: the
+ * activations of a pass live in shared memory) and contracted on the tensor cores with int8 warp MMAs against
+ * 15-bit block-fixed-point activations (blocks of 128 columns), exact int32 sums, fp32 scale epilogue.
+ * M = 1 runs the batch-1 kernel.  Format 1: one batch-1 pass per row. */
 PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, const void *packed,
                                size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                void *stream);

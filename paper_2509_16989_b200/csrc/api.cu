@@ -125,13 +125,8 @@ ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, siz
     if (m < 1 || m > PTQTP_MAX_BATCH) return PTQTP_ERR_SHAPE;
     if (!aligned16(X) || !aligned16(Y)) return PTQTP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (L.v2) {
-        for (int i = 0; i < m; ++i) {
-            s = launch_gemv2(L.l2, packed, X + (size_t)i * L.l2.k, Y + (size_t)i * L.l2.n, 0, 0, st);
-            if (s != PTQTP_OK) return s;
-        }
-        return PTQTP_OK;
-    }
+    // format 2: one batch row is fastest on the batch-1 kernel (measured); two or more go to the tensor-core kernel
+    if (L.v2) return m == 1 ? launch_gemv2(L.l2, packed, X, Y, 0, 0, st) : launch_skinny2(L.l2, packed, m, X, Y, st);
     return launch_gemm_skinny(L.l1, packed, m, X, Y, st);
 }
 

@@ -99,6 +99,8 @@ ptqtp_status launch_unpack2(const Layout2& L, const void* packed, int8_t* T1, in
                             uint16_t* a2, int32_t* dev_status, cudaStream_t st);
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
                           int depth, cudaStream_t st);
+ptqtp_status launch_skinny2(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y,
+                            cudaStream_t st);
 int sm_count();
 bool overlap_enabled();           // programmatic dependent launch of the GEMV kernels (ptqtp_set_overlap)
 

@@ -218,6 +218,32 @@ def test_gemm_skinny_matches_oracle_per_row(M, fmt):
     assert_parity(Y.cpu().numpy(), ref, np.atleast_2d(c["x"]), "M=%d" % M)
 
 
+@pytest.mark.parametrize("N,K,M", [(1, 128, 1), (5, 256, 3), (7, 1152, 4), (33, 2048, 5), (130, 3200, 8), (257, 5120, 2),
+                                   (64, 14336, 4), (1000, 6144, 7), (37, 36864, 2)])
+def test_gemm_skinny_ragged_shapes(N, K, M):
+    c = make_case(N, K, seed=300 + N, M=M)
+    packed = pack_case(c, binding.FORMAT_V2)
+    X = dev(np.atleast_2d(c["x"]))
+    Y = binding.ptqtp_gemm_skinny(packed, N, K, X, fmt=binding.FORMAT_V2)
+    torch.cuda.synchronize()
+    assert_parity(Y.cpu().numpy(), np.atleast_2d(oracle_y(c)), np.atleast_2d(c["x"]), "N=%d K=%d M=%d" % (N, K, M))
+
+
+def test_gemm_skinny_is_exact_for_integer_activations_and_matches_gemv():
+    N, K, M = 96, 4096, 6
+    c = make_case(N, K, seed=13, M=M)
+    rng = np.random.default_rng(4)
+    c["x"] = rng.integers(-3, 4, (M, K)).astype(np.float16)
+    c["alpha1"] = np.ones_like(c["alpha1"])
+    c["alpha2"] = np.full_like(c["alpha2"], 2.0)
+    exact = (c["x"].astype(np.int64) @ c["T1"].astype(np.int64).T) + 2 * (c["x"].astype(np.int64) @ c["T2"].astype(np.int64).T)
+    assert np.all(np.abs(exact) < 2048)
+    packed = pack_case(c, binding.FORMAT_V2)
+    Y = binding.ptqtp_gemm_skinny(packed, N, K, dev(c["x"]), fmt=binding.FORMAT_V2)
+    torch.cuda.synchronize()
+    assert np.array_equal(Y.cpu().numpy().astype(np.int64), exact)
+
+
 def test_gemm_skinny_config2_shape_batch8_sampled_rows():
     N, K = LLAMA3_8B_UNIQUE["gate_up"]
     c = make_case(N, K, seed=2, M=8)
