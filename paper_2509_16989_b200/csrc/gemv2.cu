@@ -116,7 +116,7 @@ constexpr int kPre = 4;                    // x loads per thread issued ahead of
 template <int D>
 __global__ void __launch_bounds__(kMaxThreads2, 1)
 gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
-             __half* __restrict__ y, int rows_cap) {
+             __half* __restrict__ y, int rows_cap, int rp_base, int rp_rem) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int nblk = L.k / kLane2;
     uint32_t* xhi = reinterpret_cast<uint32_t*>(smem);
@@ -132,8 +132,9 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     asm volatile("griddepcontrol.launch_dependents;");
 
     // this CTA's row pairs, and this warp's share of their slice units
-    const int rp0 = (int)((long long)blockIdx.x * L.nrp / gridDim.x);
-    const int rp1 = (int)((long long)(blockIdx.x + 1) * L.nrp / gridDim.x);
+    // balanced partition computed on the host: the first rp_rem CTAs take rp_base + 1 row pairs, the rest rp_base
+    const int rp0 = (int)blockIdx.x * rp_base + min((int)blockIdx.x, rp_rem);
+    const int rp1 = rp0 + rp_base + ((int)blockIdx.x < rp_rem ? 1 : 0);
     const int S = L.slices;
     const int Wc = min(S, warps);                       // slice lanes among the warps
     const int m = warps / Wc;                           // warps sharing a slice lane
@@ -307,7 +308,8 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
     cfg.attrs = attr;
     cfg.numAttrs = overlap_enabled() ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, L, static_cast<const unsigned char*>(packed),
-                                       reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap);
+                                       reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap,
+                                       L.nrp / grid, L.nrp % grid);
     if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
     return PTQTP_OK;
 }

@@ -1,0 +1,142 @@
+"""Measurements of the workloads other than the benchmark's headline step (run on a B200).
+
+    python -m paper_2509_16989_b200.report [--only 0,2,3]
+
+  0  Qwen3-0.6B up_proj 3072 x 1024, batch 1
+  2  batch sweep M in {1,...,64} of ptqtp_gemm_skinny on the 14336 x 4096 gate/up shape (and ptqtp_gemv at M = 1)
+  3  LLaMA-3-70B shapes, planes with P(0) = 0.5, batch 1 and 8
+
+(The 32-layer stack built from decomposed weights needs the CPU oracle to prepare its inputs and is therefore
+measured by tests/test_gpu_stack.py.)
+
+Every timing is a CUDA-event steady state inside a CUDA graph that walks over distinct packed buffers
+totalling more than twice the L2 size, so the planes come from HBM.  One JSON line per result.
+"""
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2509_16989_b200 import binding  # noqa: E402
+from paper_2509_16989_b200.inputs import LLAMA3_8B, LLAMA3_70B, QWEN3_0P6B_UP, make_case  # noqa: E402
+
+
+def algorithmic_bytes(N, K, M=1):
+    return N * K // 2 + 4 * N * K // 128 + 2 * M * K + 2 * M * N
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+class Timer:
+    def __init__(self):
+        self.stream = torch.cuda.Stream()
+        self.e0 = torch.cuda.Event(enable_timing=True)
+        self.e1 = torch.cuda.Event(enable_timing=True)
+        self.l2 = torch.cuda.get_device_properties(0).L2_cache_size
+
+    def copies(self, packed):
+        n = max(3, -(-(2 * self.l2 + (64 << 20)) // packed.numel()))
+        return [packed] + [packed.clone() for _ in range(n - 1)]
+
+    def steady_us(self, calls, reps=None):
+        """calls: list of zero-argument functions launching on self.stream; returns us per call."""
+        st = self.stream
+        with torch.cuda.stream(st):
+            calls[0]()
+            st.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                for c in calls:
+                    c()
+            g.replay()
+            st.synchronize()
+            reps = reps or max(3, 1500 // len(calls))
+            self.e0.record(st)
+            for _ in range(reps):
+                g.replay()
+            self.e1.record(st)
+            st.synchronize()
+        return 1e3 * self.e0.elapsed_time(self.e1) / (reps * len(calls))
+
+
+def emit(**kw):
+    print(json.dumps(kw))
+    sys.stdout.flush()
+
+
+def gemv_case(T, name, N, K, p_zero=0.4, seed=0, batches=(1,)):
+    c = make_case(N, K, seed=seed, M=max(batches), p_zero=p_zero)
+    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
+    bufs = T.copies(packed)
+    Xall = dev(np.atleast_2d(c["x"]))
+    for M in batches:
+        if M == 1:
+            x = Xall[0].contiguous()
+            y = torch.empty(N, dtype=torch.float16, device="cuda")
+            us = T.steady_us([lambda b=b: binding.ptqtp_gemv(b, N, K, x, y=y, stream=T.stream) for b in bufs])
+            call = "ptqtp_gemv"
+        else:
+            X = Xall[:M].contiguous()
+            Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+            us = T.steady_us([lambda b=b: binding.ptqtp_gemm_skinny(b, N, K, X, Y=Y, stream=T.stream) for b in bufs])
+            call = "ptqtp_gemm_skinny"
+        nb = algorithmic_bytes(N, K, M)
+        emit(workload=name, call=call, N=N, K=K, M=M, p_zero=p_zero, us=round(us, 3), gbs=round(nb / us / 1e3, 1),
+             bytes=nb, buffers=len(bufs))
+    return packed
+
+
+def config0(T):
+    N, K = QWEN3_0P6B_UP
+    gemv_case(T, "cfg0 qwen3-0.6b up_proj", N, K)
+
+
+def config2(T):
+    N, K = LLAMA3_8B["gate"]
+    c = make_case(N, K, seed=2, M=64)
+    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
+    bufs = T.copies(packed)
+    Xall = dev(c["x"])
+    for M in (1, 2, 4, 8, 16, 32, 64):
+        X = Xall[:M].contiguous()
+        Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        us = T.steady_us([lambda b=b: binding.ptqtp_gemm_skinny(b, N, K, X, Y=Y, stream=T.stream) for b in bufs])
+        nb = algorithmic_bytes(N, K, M)
+        emit(workload="cfg2 gate/up batch sweep", call="ptqtp_gemm_skinny", N=N, K=K, M=M, us=round(us, 3),
+             us_per_batch_row=round(us / M, 3), gbs=round(nb / us / 1e3, 1), bytes=nb)
+
+
+def config3(T):
+    for name, (N, K) in sorted(LLAMA3_70B.items()):
+        gemv_case(T, "cfg3 llama3-70b " + name, N, K, p_zero=0.5, seed=3, batches=(1, 8))
+        torch.cuda.empty_cache()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--only", default="0,2,3")
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise RuntimeError("needs a CUDA device")
+    binding.lib()
+    T = Timer()
+    which = set(int(v) for v in args.only.split(","))
+    if 0 in which:
+        config0(T)
+    if 2 in which:
+        config2(T)
+    if 3 in which:
+        config3(T)
+
+
+if __name__ == "__main__":
+    main()
