@@ -145,6 +145,18 @@ PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, co
                                size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                void *stream);
 
+/* Small-batch variant with a caller-provided workspace (format 2 only; PTQTP_ERR_CONFIG for format 1).
+ * Same result definition as ptqtp_gemm_skinny.  The workspace (device, 16-byte aligned, at least
+ * ptqtp_gemm_skinny_workspace_size(shape, m) bytes, contents irrelevant on entry, clobbered on return) holds X
+ * converted once to block fixed point; with it the packed planes are read from HBM exactly once for any M and
+ * K, where ptqtp_gemm_skinny needs several passes when M or K is large.  Two kernels are enqueued on `stream`.
+ * Calls that share a workspace must not overlap on the GPU.  ptqtp_gemm_skinny_workspace_size returns 0 for a
+ * bad shape, format 1 or M out of range.  Batch sweep of the benchmark spec's small-batch call list. */
+PTQTP_API size_t ptqtp_gemm_skinny_workspace_size(const ptqtp_shape *shape /* host */, int32_t m);
+PTQTP_API ptqtp_status ptqtp_gemm_skinny_ws(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
+                                  int32_t m, const uint16_t *X, uint16_t *Y, void *workspace,
+                                  size_t workspace_bytes, void *stream);
+
 /* End-to-end convenience for callers holding activations on the host: copies x_host [K] (host,
  * ideally pinned) to x_dev, runs ptqtp_gemv, copies y_dev to y_host [N]; all three enqueued on
  * `stream`, no synchronisation.  x_dev [K] and y_dev [N] are caller-owned device staging buffers. */

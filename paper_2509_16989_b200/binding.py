@@ -23,7 +23,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_SIZE, ERR_TRIT, ERR_FORMAT, ERR_CUDA, ER
 
 EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny",
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
-           "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap")
+           "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws")
 
 
 class PtqtpError(RuntimeError):
@@ -61,6 +61,10 @@ def lib():
         L.ptqtp_gemv.argtypes = [sp, vp, sz, vp, vp, vp]
         L.ptqtp_gemm_skinny.restype = ctypes.c_int
         L.ptqtp_gemm_skinny.argtypes = [sp, vp, sz, i32, vp, vp, vp]
+        L.ptqtp_gemm_skinny_workspace_size.restype = sz
+        L.ptqtp_gemm_skinny_workspace_size.argtypes = [sp, i32]
+        L.ptqtp_gemm_skinny_ws.restype = ctypes.c_int
+        L.ptqtp_gemm_skinny_ws.argtypes = [sp, vp, sz, i32, vp, vp, vp, sz, vp]
         L.ptqtp_gemv_host.restype = ctypes.c_int
         L.ptqtp_gemv_host.argtypes = [sp, vp, sz, vp, vp, vp, vp, vp]
         L.ptqtp_gemv_cfg.restype = ctypes.c_int
@@ -179,6 +183,25 @@ def ptqtp_gemm_skinny(packed, N, K, X, Y=None, stream=None, fmt=None):
                                  int(M), _dev(X, torch.float16, "X"), _dev(Y, torch.float16, "Y"),
                                  _stream_ptr(stream))
     _check(st, "ptqtp_gemm_skinny")
+    return Y
+
+
+def gemm_skinny_workspace_size(N, K, M, fmt=None):
+    return int(lib().ptqtp_gemm_skinny_workspace_size(ctypes.byref(make_shape(N, K, fmt=fmt)), int(M)))
+
+
+def ptqtp_gemm_skinny_ws(packed, N, K, X, Y=None, workspace=None, stream=None, fmt=None):
+    """ptqtp_gemm_skinny with a caller-provided workspace (uint8 CUDA tensor; allocated here if None)."""
+    shape = make_shape(N, K, fmt=fmt)
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(gemm_skinny_workspace_size(N, K, M, fmt=fmt), dtype=torch.uint8, device=X.device)
+    st = lib().ptqtp_gemm_skinny_ws(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(), int(M),
+                                    _dev(X, torch.float16, "X"), _dev(Y, torch.float16, "Y"),
+                                    _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
+    _check(st, "ptqtp_gemm_skinny_ws")
     return Y
 
 

@@ -130,6 +130,25 @@ ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, siz
     return launch_gemm_skinny(L.l1, packed, m, X, Y, st);
 }
 
+size_t ptqtp_gemm_skinny_workspace_size(const ptqtp_shape* shape, int32_t m) {
+    if (!shape_ok(shape) || shape->format != PTQTP_FORMAT_V2 || m < 1 || m > PTQTP_MAX_BATCH) return 0;
+    return skinny3_workspace_bytes(shape->k_in, m);
+}
+
+ptqtp_status ptqtp_gemm_skinny_ws(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, int32_t m,
+                                  const uint16_t* X, uint16_t* Y, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+    if (!X || !Y || !workspace) return PTQTP_ERR_NULL;
+    AnyLayout L;
+    ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
+    if (s != PTQTP_OK) return s;
+    if (m < 1 || m > PTQTP_MAX_BATCH) return PTQTP_ERR_SHAPE;
+    if (!L.v2) return PTQTP_ERR_CONFIG;
+    if (!aligned16(X) || !aligned16(Y) || !aligned16(workspace)) return PTQTP_ERR_ALIGN;
+    if (workspace_bytes < skinny3_workspace_bytes(shape->k_in, m)) return PTQTP_ERR_SIZE;
+    return launch_skinny3(L.l2, packed, m, X, Y, workspace, static_cast<cudaStream_t>(stream));
+}
+
 ptqtp_status ptqtp_gemv_host(const ptqtp_shape* shape, const void* packed, size_t packed_bytes,
                              const uint16_t* x_host, uint16_t* y_host, uint16_t* x_dev, uint16_t* y_dev,
                              void* stream) {

@@ -101,6 +101,9 @@ ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* 
                           int depth, cudaStream_t st);
 ptqtp_status launch_skinny2(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y,
                             cudaStream_t st);
+size_t skinny3_workspace_bytes(int k, int m);
+ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, void* workspace,
+                            cudaStream_t st);
 int sm_count();
 bool overlap_enabled();           // programmatic dependent launch of the GEMV kernels (ptqtp_set_overlap)
 

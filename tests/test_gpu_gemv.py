@@ -338,3 +338,47 @@ def test_overlapped_chain_keeps_stream_order(graph):
             assert np.array_equal(y.cpu().numpy().view(np.uint16), ref.view(np.uint16))
     finally:
         binding.ptqtp_set_overlap(True)
+
+
+@pytest.mark.parametrize("N,K,M", [(1, 128, 1), (5, 256, 3), (7, 1152, 4), (33, 2048, 5), (130, 3200, 8), (257, 5120, 12),
+                                   (64, 14336, 16), (1000, 6144, 33), (37, 36864, 2), (192, 3072, 64), (2400, 4096, 9)])
+def test_gemm_skinny_ws_matches_oracle(N, K, M):
+    c = make_case(N, K, seed=400 + N, M=M)
+    packed = pack_case(c, binding.FORMAT_V2)
+    X = dev(np.atleast_2d(c["x"]))
+    need = binding.gemm_skinny_workspace_size(N, K, M)
+    assert need > 0
+    ws = torch.full((need + 64,), 0xA5, dtype=torch.uint8, device="cuda")       # dirty workspace + guard band
+    Y = binding.ptqtp_gemm_skinny_ws(packed, N, K, X, workspace=ws[:need], fmt=binding.FORMAT_V2)
+    torch.cuda.synchronize()
+    assert bool((ws[need:] == 0xA5).all())
+    ref = np.atleast_2d(oracle_y(c))
+    assert_parity(Y.cpu().numpy(), ref, np.atleast_2d(c["x"]), "N=%d K=%d M=%d" % (N, K, M))
+    # a second call on the same (now used) workspace with other activations must not see the first call's
+    c2 = make_case(N, K, seed=900 + N, M=M)
+    Y2 = binding.ptqtp_gemm_skinny_ws(packed, N, K, dev(np.atleast_2d(c2["x"])), workspace=ws[:need], fmt=binding.FORMAT_V2)
+    torch.cuda.synchronize()
+    assert_parity(Y2.cpu().numpy(), np.atleast_2d(oracle_y(dict(c, x=c2["x"]))), np.atleast_2d(c2["x"]), "second call")
+
+
+def test_gemm_skinny_ws_argument_checks_and_exactness():
+    N, K, M = 96, 4096, 6
+    c = make_case(N, K, seed=14, M=M)
+    rng = np.random.default_rng(5)
+    c["x"] = rng.integers(-3, 4, (M, K)).astype(np.float16)
+    c["alpha1"] = np.ones_like(c["alpha1"])
+    c["alpha2"] = np.full_like(c["alpha2"], 2.0)
+    exact = (c["x"].astype(np.int64) @ c["T1"].astype(np.int64).T) + 2 * (c["x"].astype(np.int64) @ c["T2"].astype(np.int64).T)
+    packed = pack_case(c, binding.FORMAT_V2)
+    Y = binding.ptqtp_gemm_skinny_ws(packed, N, K, dev(c["x"]), fmt=binding.FORMAT_V2)
+    torch.cuda.synchronize()
+    assert np.array_equal(Y.cpu().numpy().astype(np.int64), exact)
+    small = torch.empty(binding.gemm_skinny_workspace_size(N, K, M) - 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.PtqtpError) as e:
+        binding.ptqtp_gemm_skinny_ws(packed, N, K, dev(c["x"]), workspace=small, fmt=binding.FORMAT_V2)
+    assert e.value.status == binding.ERR_SIZE
+    assert binding.gemm_skinny_workspace_size(N, K, 65) == 0 and binding.gemm_skinny_workspace_size(N, K, M, fmt=1) == 0
+    p1 = pack_case(c, binding.FORMAT_V1)
+    with pytest.raises(binding.PtqtpError) as e:
+        binding.ptqtp_gemm_skinny_ws(p1, N, K, dev(c["x"]), workspace=small, fmt=binding.FORMAT_V1)
+    assert e.value.status == binding.ERR_CONFIG
