@@ -101,6 +101,7 @@ typedef struct {
 #define PTQTP_FORMAT_V2 2
 #define PTQTP_HEADER_BYTES 256
 #define PTQTP_MAX_BATCH 64
+#define PTQTP_STATIC_WORKSPACE_BYTES (512 * 1024)
 
 /* Size in bytes of the packed blob for `shape` (header and padding included); 0 on a bad shape.
  * Storage model: Appendix B "Memory Saving" (2 bits per trit, fp16 scales per group). */
@@ -156,6 +157,28 @@ PTQTP_API size_t ptqtp_gemm_skinny_workspace_size(const ptqtp_shape *shape /* ho
 PTQTP_API ptqtp_status ptqtp_gemm_skinny_ws(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                                   int32_t m, const uint16_t *X, uint16_t *Y, void *workspace,
                                   size_t workspace_bytes, void *stream);
+
+/* ptqtp_gemm_skinny_ws for callers that cannot hand over a workspace.  (The paper has no counterpart: this
+ * entry point exists for the library's users, not for the method.)
+ * Who needs it: code that runs where device memory cannot be allocated -- a plug-in or C caller inside a host
+ * process whose framework already owns all of the GPU's memory through its own pool and exposes no allocator,
+ * code on a latency-critical decode path where cudaMalloc/cudaFree would stall the whole device, and code
+ * that must not call allocating CUDA routines at all at that point (for instance while other threads are
+ * capturing streams).  The workspace is a fixed array of PTQTP_STATIC_WORKSPACE_BYTES (512 KiB) in device
+ * memory that belongs to the library: every GPU that loads the library carries it until the process exits.
+ * This call never calls cudaMalloc, cudaFree or any allocating library routine; the caller still owns
+ * packed, X and Y.
+ * Limits: the (K, M) pair must satisfy ptqtp_gemm_skinny_workspace_size(shape, m) <=
+ * PTQTP_STATIC_WORKSPACE_BYTES (e.g. M <= 8 up to K = 28672, M <= 16 up to K = 14336, M <= 64 up to K = 3072);
+ * otherwise PTQTP_ERR_SIZE is returned and nothing is launched.  Format 2 only (PTQTP_ERR_CONFIG for format 1).
+ * The first call on each device looks up the array's device address (with that device current, no
+ * allocation); make that first call outside any stream capture.
+ * All calls on a device share the one array.  It keeps the previous call's contents; each call rewrites every
+ * byte it later reads (padding included), so stale contents are harmless, but two calls that overlap on the
+ * GPU (different streams, or the same call from two threads) race on it: serialise them. */
+PTQTP_API ptqtp_status ptqtp_gemm_skinny_static(const ptqtp_shape *shape /* host */, const void *packed,
+                                      size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
+                                      void *stream);
 
 /* End-to-end convenience for callers holding activations on the host: copies x_host [K] (host,
  * ideally pinned) to x_dev, runs ptqtp_gemv, copies y_dev to y_host [N]; all three enqueued on

@@ -23,7 +23,8 @@ OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_SIZE, ERR_TRIT, ERR_FORMAT, ERR_CUDA, ER
 
 EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny",
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
-           "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws")
+           "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws",
+           "ptqtp_gemm_skinny_static")
 
 
 class PtqtpError(RuntimeError):
@@ -65,6 +66,8 @@ def lib():
         L.ptqtp_gemm_skinny_workspace_size.argtypes = [sp, i32]
         L.ptqtp_gemm_skinny_ws.restype = ctypes.c_int
         L.ptqtp_gemm_skinny_ws.argtypes = [sp, vp, sz, i32, vp, vp, vp, sz, vp]
+        L.ptqtp_gemm_skinny_static.restype = ctypes.c_int
+        L.ptqtp_gemm_skinny_static.argtypes = [sp, vp, sz, i32, vp, vp, vp]
         L.ptqtp_gemv_host.restype = ctypes.c_int
         L.ptqtp_gemv_host.argtypes = [sp, vp, sz, vp, vp, vp, vp, vp]
         L.ptqtp_gemv_cfg.restype = ctypes.c_int
@@ -202,6 +205,23 @@ def ptqtp_gemm_skinny_ws(packed, N, K, X, Y=None, workspace=None, stream=None, f
                                     _dev(X, torch.float16, "X"), _dev(Y, torch.float16, "Y"),
                                     _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream_ptr(stream))
     _check(st, "ptqtp_gemm_skinny_ws")
+    return Y
+
+
+STATIC_WORKSPACE_BYTES = 512 * 1024
+
+
+def ptqtp_gemm_skinny_static(packed, N, K, X, Y, stream=None, fmt=None):
+    """ptqtp_gemm_skinny_ws on the library's own fixed workspace: for callers that cannot allocate device memory.
+
+    Y must be passed in (this wrapper allocates nothing either).  Raises PtqtpError(ERR_SIZE) when
+    gemm_skinny_workspace_size(N, K, M) exceeds STATIC_WORKSPACE_BYTES.  Calls share one array per device:
+    do not let two of them overlap on the GPU."""
+    shape = make_shape(N, K, fmt=fmt)
+    st = lib().ptqtp_gemm_skinny_static(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
+                                        int(X.shape[0]), _dev(X, torch.float16, "X"), _dev(Y, torch.float16, "Y"),
+                                        _stream_ptr(stream))
+    _check(st, "ptqtp_gemm_skinny_static")
     return Y
 
 

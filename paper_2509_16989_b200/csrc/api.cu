@@ -149,6 +149,22 @@ ptqtp_status ptqtp_gemm_skinny_ws(const ptqtp_shape* shape, const void* packed, 
     return launch_skinny3(L.l2, packed, m, X, Y, workspace, static_cast<cudaStream_t>(stream));
 }
 
+ptqtp_status ptqtp_gemm_skinny_static(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, int32_t m,
+                                      const uint16_t* X, uint16_t* Y, void* stream) {
+    if (!X || !Y) return PTQTP_ERR_NULL;
+    AnyLayout L;
+    ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
+    if (s != PTQTP_OK) return s;
+    if (m < 1 || m > PTQTP_MAX_BATCH) return PTQTP_ERR_SHAPE;
+    if (!L.v2) return PTQTP_ERR_CONFIG;
+    if (!aligned16(X) || !aligned16(Y)) return PTQTP_ERR_ALIGN;
+    if (skinny3_workspace_bytes(shape->k_in, m) > (size_t)PTQTP_STATIC_WORKSPACE_BYTES) return PTQTP_ERR_SIZE;
+    void* workspace = nullptr;
+    s = static_workspace_address(&workspace);
+    if (s != PTQTP_OK) return s;
+    return launch_skinny3(L.l2, packed, m, X, Y, workspace, static_cast<cudaStream_t>(stream));
+}
+
 ptqtp_status ptqtp_gemv_host(const ptqtp_shape* shape, const void* packed, size_t packed_bytes,
                              const uint16_t* x_host, uint16_t* y_host, uint16_t* x_dev, uint16_t* y_dev,
                              void* stream) {

@@ -16,7 +16,13 @@
 //   * The main kernel issues its first code copies before griddepcontrol.wait, i.e. while the conversion kernel
 //     (or whatever precedes it on the stream) is still running.
 #include <cuda_fp16.h>
+#include <mutex>
 #include "ptqtp_internal.h"
+
+// Workspace of ptqtp_gemm_skinny_static: a fixed array in device memory, owned by the library, present on every
+// GPU that loads it until the process exits.  In host code this name is only a handle for the runtime (its
+// device address comes from cudaGetSymbolAddress); device code may name it directly.
+static __device__ __align__(256) unsigned char g_static_workspace[PTQTP_STATIC_WORKSPACE_BYTES];
 
 namespace ptqtp {
 
@@ -318,6 +324,26 @@ ptqtp_status launch3(const Layout2& L, const void* packed, const unsigned char* 
 }  // namespace
 
 size_t skinny3_workspace_bytes(int k, int m) { return ws3_layout(k, m).total; }
+
+// Device address of the library-owned workspace on the current device.  Looked up once per device, with that
+// device current, and cached; nothing is allocated.
+ptqtp_status static_workspace_address(void** out) {
+    static std::mutex lock;
+    static void* cached[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return PTQTP_ERR_CONFIG;
+    std::lock_guard<std::mutex> guard(lock);
+    if (!cached[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_workspace);
+        if (e != cudaSuccess || !p) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+        cached[dev] = p;
+    }
+    *out = cached[dev];
+    return PTQTP_OK;
+}
 
 ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, void* workspace,
                             cudaStream_t st) {
