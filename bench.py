@@ -34,6 +34,9 @@ WORKLOAD = "llama3-8b decode linears (q,k,v,o 4096x4096|1024x4096, gate/up 14336
 MATRICES = ("q", "k", "v", "o", "gate", "up", "down")
 UNIQUE_OF = {"q": "qo", "o": "qo", "k": "kv", "v": "kv", "gate": "gate_up", "up": "gate_up", "down": "down"}
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes in the ncu capture of the 14336x4096 launch of
+# the current GEMV kernel (profiles/gemv2_gate_up_14336x4096.md); set to None when the kernel changes
+DRAM_TRAFFIC_RATIO = 31234048.0 / 31232000.0
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -423,7 +426,8 @@ def run_gpu(args):
         "weight_gbs": STEP_WEIGHT_BYTES / (ms_per_step * 1e-3) / 1e9,
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": "of " + peak_kind, "traffic": None,
+                     "peak_kind": "of " + peak_kind,
+                     "traffic": None if DRAM_TRAFFIC_RATIO is None else DRAM_TRAFFIC_RATIO * STEP_BYTES / 7.0,
                      "kernel": "gemv2_kernel (7 launches per step; mean over the step)",
                      "bytes_per_launch_mean": STEP_BYTES / 7.0, "us_per_launch_mean": 1e3 * ms_per_step / 7.0},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
