@@ -49,7 +49,7 @@ __device__ __forceinline__ void cp_wait_all() { asm volatile("cp.async.wait_grou
 
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -134,19 +134,22 @@ convert3_kernel(const __half* __restrict__ X, unsigned char* __restrict__ ws, in
 template <int NTT>
 __global__ void __launch_bounds__(kMaxWarps3 * 32, 1)
 skinny3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const unsigned char* __restrict__ ws,
-               __half* __restrict__ Y, int m, int q_base, int q_rem) {
+               __half* __restrict__ Y, int m, int q_base, int q_rem, int depth) {
     constexpr int NTG = NTT < 4 ? NTT : 4;
     constexpr int NG = NTT / NTG;
-    constexpr int kTileBytes = 8 * NTG * kTileRow;
+    constexpr int kTileRows = 8 * NTG * kTileRow;                       // activation rows of a tile
+    constexpr int kTileBytes = kTileRows + 4 * NTG * 64;                // + (2^-s, sum X) of 4 NTG batch rows x 8 groups
     extern __shared__ __align__(16) unsigned char smem[];
     asm volatile("griddepcontrol.launch_dependents;");
 
-    const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the last warp only copies activation tiles; the others ("compute warps") stream and contract codes
+    const int warps = (blockDim.x >> 5) - 1, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool loader = warp == warps;
     const int g = lane >> 2, tig = lane & 3, u = g & 3, plane = g >> 2;
     const Ws3 w = ws3_layout(L.k, m);
     const int halves = w.halves, ngroups = L.k / kGroup;
     unsigned char* tile = smem;                                          // [2][8 NTG rows][kTileRow]
-    unsigned char* ring = smem + 2 * kTileBytes + (size_t)warp * 2 * kQuadSlot;
+    unsigned char* ring = smem + 2 * kTileBytes + (size_t)(loader ? 0 : warp) * depth * kQuadSlot;
     const int2* meta = reinterpret_cast<const int2*>(ws + w.meta_off);
 
     // this CTA's quads (balanced partition from the host) and the rounds needed to give every quad a warp
@@ -174,23 +177,46 @@ skinny3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const unsign
             if (lane < Ah / 2) cp8(d + kScaleChunk * 16 + lane * 8, src + A * 64 + (l0 / 2 + lane) * 8);
         }
     };
-    // activation tile of (half slice, n-tile group) -> tile buffer; all threads share the copy
+    // activation tile of (half slice, n-tile group) -> tile buffer, copied by the loader warp
     auto issue_tile = [&](int hs, int ng, int buf) {
         const unsigned char* src = ws + ((size_t)hs * 2 * w.m_pad + 8 * NTG * ng) * kHalf;
         unsigned char* dst = tile + buf * kTileBytes;
-        for (int c = threadIdx.x; c < 8 * NTG * (kHalf / 16); c += blockDim.x)
+        for (int c = lane; c < 8 * NTG * (kHalf / 16); c += 32)
             cp16(dst + (c >> 6) * kTileRow + (c & 63) * 16, src + (size_t)c * 16);
+        // the records of the tile's batch rows for the (up to) 8 groups of the half slice
+        for (int c = lane; c < 4 * NTG * 8; c += 32) {
+            const int row = c >> 3, gi = hs * 8 + (c & 7);
+            if (gi < ngroups) cp8(dst + kTileRows + c * 8, meta + (size_t)(4 * NTG * ng + row) * ngroups + gi);
+        }
     };
 
-    const int steps = rounds * halves * NG;
-    const bool has0 = warp < nq_cta;
-    if (has0) issue_codes(q0 + warp, 0, 0);
-    cp_commit();
+    const int steps = rounds * halves * NG;              // activation-tile steps
+    const int code_steps = rounds * halves;              // (round, half slice) pairs: one ring slot each
+    // codes of code step cs for this warp (if it has a quad in that round) -> ring slot cs % depth
+    auto issue_code_step = [&](int cs) {
+        if (!loader && cs < code_steps) {
+            const int r = cs / halves, hs = cs - r * halves;
+            const int ql = r * warps + warp;
+            if (ql < nq_cta) issue_codes(q0 + ql, hs, cs % depth);
+        }
+        cp_commit();
+    };
+    // wait until at most depth - 2 of this thread's copy groups are pending: the codes of the next code step have
+    // landed, younger ones may still be in flight
+    auto wait_codes = [&]() {
+        if (depth >= 3) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else cp_wait_all();
+    };
+    for (int d = 0; d < depth - 1; ++d) issue_code_step(d);
     // everything above reads only the packed planes; the workspace and Y belong to the stream order
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (steps > 0) issue_tile(0, 0, 0);
-    cp_commit();
-    cp_wait_all();
+    if (loader) {
+        if (steps > 0) issue_tile(0, 0, 0);
+        cp_commit();
+        cp_wait_all();
+    } else {
+        wait_codes();
+    }
     __syncthreads();
 
     const uint32_t maskA = 0x03030303u << (2 * plane), maskB = maskA << 4;       // fields plane and 2 + plane
@@ -198,10 +224,10 @@ skinny3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const unsign
     const int shA = 2 * plane, shB = shA + 4;
     const uint32_t alpha_sel = plane ? 0x7632u : 0x5410u;
 
-    int t = 0, slot = 0;
+    int t = 0, cs = 0, slot = 0;
     for (int r = 0; r < rounds; ++r) {
         const int ql = r * warps + warp;                 // this warp's quad of the round, if any
-        const bool has = ql < nq_cta;
+        const bool has = !loader && ql < nq_cta;
         const int q = q0 + ql;
         float yA[NTT], yB[NTT];
 #pragma unroll
@@ -210,27 +236,23 @@ skinny3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const unsign
             const int sl = hs >> 1, l0 = (hs & 1) * 16;
             const int A = sl == L.slices - 1 ? L.last_active : 32;
             const int groups_here = min(16, A - l0) / 2;
-            // prefetch this warp's codes of the next (round, half slice) into the other slot
-            {
-                int nhs = hs + 1, nql = ql;
-                if (nhs == halves) { nhs = 0; nql += warps; }
-                if (nql < nq_cta) issue_codes(q0 + nql, nhs, slot ^ 1);
-            }
+            // keep depth - 1 code steps in flight
+            if (!loader) issue_code_step(cs + depth - 1);
 #pragma unroll
             for (int ng = 0; ng < NG; ++ng) {
-                // prefetch the next step's activation tile into the other buffer
-                {
+                if (loader) {                            // the next step's activation tile into the other buffer
                     int nng = ng + 1, nhs = hs;
                     if (nng == NG) { nng = 0; if (++nhs == halves) nhs = 0; }
                     if (t + 1 < steps) issue_tile(nhs, nng, (t + 1) & 1);
+                    cp_commit();
                 }
-                cp_commit();
                 if (has) {
                     const unsigned char* unit = ring + slot * kQuadSlot + u * (kSU * 16);
                     const unsigned char* cptr = unit + (tig * kSI) * 16;
                     const unsigned char* sptr = unit + kScaleChunk * 16;
                     const unsigned char* xptr = tile + (t & 1) * kTileBytes + g * kTileRow + 16 * tig;
-                    const int2* mptr = meta + (size_t)(4 * NTG * ng + tig) * ngroups + hs * 8;
+                    const unsigned char* mptr = tile + (t & 1) * kTileBytes + kTileRows + tig * 64;
+#pragma unroll 2
                     for (int gl = 0; gl < groups_here; ++gl) {       // one 128-column scale group per iteration
                         int c[NTG][4];
 #pragma unroll
@@ -253,7 +275,7 @@ skinny3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const unsign
                         const float wA = al.x * kA, wB = al.y * kB;
 #pragma unroll
                         for (int nt = 0; nt < NTG; ++nt) {
-                            const int2 rec = __ldg(mptr + (size_t)(4 * nt) * ngroups);      // batch row 4 (NTG ng + nt) + tig
+                            const int2 rec = *reinterpret_cast<const int2*>(mptr + nt * 256);   // batch row 4 (NTG ng + nt) + tig
                             const float cm = __int_as_float(rec.x);
                             const int QA = (c[nt][0] << 8) + c[nt][1] - (rec.y << shA);
                             const int QB = (c[nt][2] << 8) + c[nt][3] - (rec.y << shB);
@@ -263,15 +285,16 @@ skinny3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const unsign
                         cptr += 32;
                         sptr += 8;
                         xptr += 128;
-                        mptr += 1;
+                        mptr += 8;
                     }
                 }
                 // the next tile and the next codes have landed and everybody is done with this step's tile
-                cp_wait_all();
+                if (loader) cp_wait_all(); else wait_codes();
                 __syncthreads();
                 ++t;
             }
-            slot ^= 1;
+            ++cs;
+            slot = slot + 1 == depth ? 0 : slot + 1;
         }
         // the two planes of a row are 16 lanes apart; lanes 0-15 write the quad's rows for batch rows 4 nt + tig
 #pragma unroll
@@ -287,16 +310,17 @@ skinny3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const unsign
     }
 }
 
-size_t smem3(int ntt, int warps) {
+size_t smem3(int ntt, int compute_warps, int depth) {
     const int ntg = ntt < 4 ? ntt : 4;
-    return (size_t)2 * 8 * ntg * kTileRow + (size_t)warps * 2 * kQuadSlot;
+    return (size_t)2 * (8 * ntg * kTileRow + 4 * ntg * 64) + (size_t)compute_warps * depth * kQuadSlot;
 }
 
 template <int NTT>
 ptqtp_status launch3(const Layout2& L, const void* packed, const unsigned char* ws, uint16_t* Y, int m, int grid,
                      int warps, int nq, cudaStream_t st) {
     auto kern = skinny3_kernel<NTT>;
-    const size_t smem = smem3(NTT, warps);
+    const int depth = smem3(NTT, warps, 3) <= 227 * 1024 ? 3 : 2;         // ring slots per compute warp
+    const size_t smem = smem3(NTT, warps, depth);
     static thread_local size_t configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
@@ -307,7 +331,7 @@ ptqtp_status launch3(const Layout2& L, const void* packed, const unsigned char* 
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(warps * 32);
+    cfg.blockDim = dim3((warps + 1) * 32);                               // + the tile loader warp
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -316,7 +340,7 @@ ptqtp_status launch3(const Layout2& L, const void* packed, const unsigned char* 
     cfg.attrs = attr;
     cfg.numAttrs = overlap_enabled() ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, L, static_cast<const unsigned char*>(packed), ws,
-                                       reinterpret_cast<__half*>(Y), m, nq / grid, nq % grid);
+                                       reinterpret_cast<__half*>(Y), m, nq / grid, nq % grid, depth);
     if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
     return PTQTP_OK;
 }
@@ -354,12 +378,12 @@ ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const u
     convert3_kernel<<<(unsigned)(tasks / 256), 256, 0, st>>>(reinterpret_cast<const __half*>(X), ws, L.k, m);
     ptqtp_status s = check_launch();
     if (s != PTQTP_OK) return s;
-    // kernel 2: one CTA per SM, one quad per warp and round; as many warps as the CTA with most quads needs
+    // kernel 2: one CTA per SM, one quad per compute warp and round; as many as the CTA with most quads needs
     const int nq = (L.nrp + 3) / 4;
     const int grid = min(sm_count(), nq);
     const int per_cta = (nq + grid - 1) / grid;
-    const int rounds = (per_cta + kMaxWarps3 - 1) / kMaxWarps3;
-    const int warps = max(4, (per_cta + rounds - 1) / rounds);            // idle warps still help copying tiles
+    const int rounds = (per_cta + kMaxWarps3 - 2) / (kMaxWarps3 - 1);     // one of the 16 warps only loads tiles
+    const int warps = (per_cta + rounds - 1) / rounds;                    // compute warps
     switch (w.m_pad / 4) {
         case 1: return launch3<1>(L, packed, ws, Y, m, grid, warps, nq, st);
         case 2: return launch3<2>(L, packed, ws, Y, m, grid, warps, nq, st);

@@ -89,6 +89,12 @@ def gemv_case(T, name, N, K, p_zero=0.4, seed=0, batches=(1,)):
             Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
             us = T.steady_us([lambda b=b: binding.ptqtp_gemm_skinny(b, N, K, X, Y=Y, stream=T.stream) for b in bufs])
             call = "ptqtp_gemm_skinny"
+            ws = torch.empty(binding.gemm_skinny_workspace_size(N, K, M), dtype=torch.uint8, device="cuda")
+            us_ws = T.steady_us([lambda b=b: binding.ptqtp_gemm_skinny_ws(b, N, K, X, Y=Y, workspace=ws, stream=T.stream)
+                                 for b in bufs])
+            nb = algorithmic_bytes(N, K, M)
+            emit(workload=name, call="ptqtp_gemm_skinny_ws", N=N, K=K, M=M, p_zero=p_zero, us=round(us_ws, 3),
+                 gbs=round(nb / us_ws / 1e3, 1), bytes=nb, buffers=len(bufs))
         nb = algorithmic_bytes(N, K, M)
         emit(workload=name, call=call, N=N, K=K, M=M, p_zero=p_zero, us=round(us, 3), gbs=round(nb / us / 1e3, 1),
              bytes=nb, buffers=len(bufs))
@@ -112,6 +118,11 @@ def config2(T):
         us = T.steady_us([lambda b=b: binding.ptqtp_gemm_skinny(b, N, K, X, Y=Y, stream=T.stream) for b in bufs])
         nb = algorithmic_bytes(N, K, M)
         emit(workload="cfg2 gate/up batch sweep", call="ptqtp_gemm_skinny", N=N, K=K, M=M, us=round(us, 3),
+             us_per_batch_row=round(us / M, 3), gbs=round(nb / us / 1e3, 1), bytes=nb)
+        ws = torch.empty(binding.gemm_skinny_workspace_size(N, K, M), dtype=torch.uint8, device="cuda")
+        us = T.steady_us([lambda b=b: binding.ptqtp_gemm_skinny_ws(b, N, K, X, Y=Y, workspace=ws, stream=T.stream)
+                          for b in bufs])
+        emit(workload="cfg2 gate/up batch sweep", call="ptqtp_gemm_skinny_ws", N=N, K=K, M=M, us=round(us, 3),
              us_per_batch_row=round(us / M, 3), gbs=round(nb / us / 1e3, 1), bytes=nb)
 
 
