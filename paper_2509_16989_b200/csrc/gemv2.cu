@@ -104,9 +104,12 @@ __device__ __forceinline__ void convert_x8(uint4 raw, int base, bool valid, uint
         hw[w] = __byte_perm(hi01, hi23, 0x5410);
     }
     if (valid) {
+        // the four 16-byte chunks of a block are stored permuted (chunk v at v ^ swz) so that the lanes of a warp,
+        // which each read a whole block with 128-bit loads, do not collide on shared-memory banks
         const int blk = base >> 6, tt = (base >> 3) & 7;
-        *reinterpret_cast<uint2*>(xhi + blk * 16 + 2 * tt) = make_uint2(hw[0], hw[1]);
-        *reinterpret_cast<uint2*>(xlo + blk * 16 + 2 * tt) = make_uint2(lw[0], lw[1]);
+        const int pos = blk * 16 + (((tt >> 1) ^ ((blk >> 1) & 3)) << 2) + ((tt & 1) << 1);
+        *reinterpret_cast<uint2*>(xhi + pos) = make_uint2(hw[0], hw[1]);
+        *reinterpret_cast<uint2*>(xlo + pos) = make_uint2(lw[0], lw[1]);
         if (tt == 0) meta[blk] = make_int2((int)((uint32_t)(127 - s) << 23), sum);
     }
 }
@@ -214,8 +217,9 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
         const int blk = sl * 32 + (live ? lane : 0);
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
-            const uint4 a = *reinterpret_cast<const uint4*>(xhi + blk * 16 + 4 * v);
-            const uint4 b = *reinterpret_cast<const uint4*>(xlo + blk * 16 + 4 * v);
+            const int pos = blk * 16 + ((v ^ ((blk >> 1) & 3)) << 2);
+            const uint4 a = *reinterpret_cast<const uint4*>(xhi + pos);
+            const uint4 b = *reinterpret_cast<const uint4*>(xlo + pos);
             xh[4 * v] = a.x; xh[4 * v + 1] = a.y; xh[4 * v + 2] = a.z; xh[4 * v + 3] = a.w;
             xl[4 * v] = b.x; xl[4 * v + 1] = b.y; xl[4 * v + 2] = b.z; xl[4 * v + 3] = b.w;
         }
