@@ -212,6 +212,12 @@ PTQTP_API const char *ptqtp_status_string(ptqtp_status status);
 /* The cudaError_t (as int) behind the calling thread's most recent PTQTP_ERR_CUDA, else 0. */
 PTQTP_API int ptqtp_last_cuda_error(void);
 
+/* Device-side health of the batch-1 kernel on the current device.  The format-2 GEMV streams the packed planes
+ * with bulk copies and waits for each with a bounded number of polls; if a wait ever gives up, the kernel
+ * writes NaN to the rows it could not finish, records PTQTP_ERR_CUDA in a device word and still terminates.
+ * This call enqueues a copy of that word (0 = healthy) to *status_host on `stream`; read it after syncing. */
+PTQTP_API ptqtp_status ptqtp_kernel_status(int32_t *status_host /* host */, void *stream);
+
 /* Overlap of consecutive GEMV calls on one stream (process-wide switch, on by default; returns the old
  * value).  When on, format-2 GEMV kernels are launched with programmatic stream serialization: a call may
  * begin reading its `packed` blob while the GEMV call directly before it on the stream is still draining;

@@ -24,7 +24,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_SIZE, ERR_TRIT, ERR_FORMAT, ERR_CUDA, ER
 EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny",
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
            "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws",
-           "ptqtp_gemm_skinny_static")
+           "ptqtp_gemm_skinny_static", "ptqtp_kernel_status")
 
 
 class PtqtpError(RuntimeError):
@@ -78,6 +78,8 @@ def lib():
         L.ptqtp_status_string.argtypes = [ctypes.c_int]
         L.ptqtp_last_cuda_error.restype = ctypes.c_int
         L.ptqtp_version.restype = ctypes.c_int
+        L.ptqtp_kernel_status.restype = ctypes.c_int
+        L.ptqtp_kernel_status.argtypes = [ctypes.POINTER(ctypes.c_int32), vp]
         L.ptqtp_set_overlap.restype = ctypes.c_int
         L.ptqtp_set_overlap.argtypes = [ctypes.c_int]
         _lib = L
@@ -237,6 +239,16 @@ def ptqtp_gemv_host(packed, N, K, x_host, y_host, x_dev, y_dev, stream=None, fmt
                                _stream_ptr(stream))
     _check(st, "ptqtp_gemv_host")
     return y_host
+
+
+def ptqtp_kernel_status(stream=None):
+    """Device-side health word of the batch-1 kernel (0 = healthy); synchronises the stream to read it."""
+    out = ctypes.c_int32(-1)
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    _check(lib().ptqtp_kernel_status(ctypes.byref(out), ctypes.c_void_p(stream.cuda_stream)), "ptqtp_kernel_status")
+    stream.synchronize()
+    return int(out.value)
 
 
 def ptqtp_set_overlap(enabled):

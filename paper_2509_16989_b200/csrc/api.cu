@@ -224,6 +224,11 @@ const char* ptqtp_status_string(ptqtp_status status) {
 
 int ptqtp_last_cuda_error(void) { return g_last_cuda_error; }
 
+ptqtp_status ptqtp_kernel_status(int32_t* status_host, void* stream) {
+    if (!status_host) return PTQTP_ERR_NULL;
+    return copy_gemv2_status(status_host, static_cast<cudaStream_t>(stream));
+}
+
 int ptqtp_set_overlap(int enabled) {
     const int old = g_overlap;
     g_overlap = enabled ? 1 : 0;

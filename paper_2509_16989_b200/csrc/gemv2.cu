@@ -17,8 +17,11 @@
 //     four accumulator pairs (2 rows x 2 planes) see one scale group half and get the group's scales
 //     (the method's only multiplies) in an fp32 epilogue.
 //   * Each warp streams its slice units (2048 code bytes + 128 scale bytes, contiguous in HBM) through a
-//     private shared-memory ring with cp.async, several units in flight, issued before x is staged.  A lane
-//     reads back only bytes it copied itself, so no barrier is needed inside the stream.
+//     private shared-memory ring: one bulk copy (cp.async.bulk, no multicast) per unit, issued by lane 0 and
+//     completed on an mbarrier, several units in flight, the first ones issued before x is fetched.  Bulk
+//     copies cost no load/store-unit time, which matters because the whole CTA waits for the fetch of x.
+//     Every wait on an mbarrier is bounded: if one gives up the warp writes NaN rows, records an error in a
+//     device status word (ptqtp_kernel_status) and still runs to the end.
 //   * Rows are reduced over the lanes by shuffles, over the slices through shared memory in a fixed order
 //     (deterministic), rounded once to fp16.
 #include <cuda_fp16.h>
@@ -26,23 +29,37 @@
 
 namespace ptqtp {
 
+// Device-side status of the GEMV kernel: set when a bounded wait for a bulk copy gave up.
+__device__ int g_gemv2_status = 0;
+
 namespace {
 
-constexpr int kSlot = 2048 + 256;          // ring slot: 128 atoms of 16 B + one 8-byte scale quad per lane
 constexpr int kMaxWarps2 = 16;
 constexpr int kMaxThreads2 = kMaxWarps2 * 32;
+constexpr int kSpinLimit = 1 << 22;             // polls of an mbarrier before a wait gives up
+constexpr int kSpinLimitAfterFailure = 1 << 8;
 
-__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
-    const unsigned d = (unsigned)__cvta_generic_to_shared(dst_smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async8(void* dst_smem, const void* src) {
-    const unsigned d = (unsigned)__cvta_generic_to_shared(dst_smem);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(src) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bulk copy global -> this CTA's shared memory, completion counted in bytes on an mbarrier (no multicast).
+__device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
 
 // d = c + sum_b u8(a.b) * s8(x.b)   and   d = c + sum_b u8(a.b) * u8(x.b)
 __device__ __forceinline__ int dot_us(uint32_t a, uint32_t x, int c) {
@@ -116,6 +133,20 @@ __device__ __forceinline__ void convert_x8(uint4 raw, int base, bool valid, uint
 
 constexpr int kPre = 4;                    // x loads per thread issued ahead of the weight stream
 
+// Shared memory: x as two byte planes and block records, the per-slice partial sums, one mbarrier per ring slot,
+// then the ring (one slice unit, kUnit2 bytes, per slot; D slots per warp).
+struct Smem2 {
+    size_t partial_off, bar_off, ring_off, total;
+};
+__host__ __device__ inline Smem2 smem_layout2(int k, int slices, int rows_cap, int warps, int depth) {
+    Smem2 m;
+    m.partial_off = (size_t)(k / kLane2) * 136;
+    m.bar_off = (m.partial_off + (size_t)rows_cap * slices * 4 + 7) / 8 * 8;
+    m.ring_off = (m.bar_off + (size_t)warps * depth * 8 + 15) / 16 * 16;
+    m.total = m.ring_off + (size_t)warps * depth * kUnit2;
+    return m;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kMaxThreads2, 1)
 gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
@@ -125,11 +156,12 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     uint32_t* xhi = reinterpret_cast<uint32_t*>(smem);
     uint32_t* xlo = xhi + nblk * 16;
     int2* meta = reinterpret_cast<int2*>(xlo + nblk * 16);
-    float* partial = reinterpret_cast<float*>(meta + nblk);                 // [rows_cap][slices]
     const int warps = blockDim.x >> 5;
-    const size_t ring_off = ((size_t)nblk * 136 + (size_t)rows_cap * L.slices * 4 + 15) / 16 * 16;
+    const Smem2 sm = smem_layout2(L.k, L.slices, rows_cap, warps, D);
+    float* partial = reinterpret_cast<float*>(smem + sm.partial_off);       // [rows_cap][slices]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned char* ring_lane = smem + ring_off + (size_t)warp * D * kSlot + lane * 16;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bar_off) + warp * D;
+    unsigned char* ring = smem + sm.ring_off + (size_t)warp * D * kUnit2;
 
     // Let the next kernel on the stream start its own weight prefetch while this one drains.
     asm volatile("griddepcontrol.launch_dependents;");
@@ -148,37 +180,36 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     const unsigned char* codes = packed + L.codes_off + (size_t)(rp0 + wi) * L.strip;
     const size_t rp_stride = (size_t)m * L.strip;
 
-    // prefetch cursor: slice pass pt, row pair pj, source of the next unit, ring slot offset
+    if (lane == 0) {
+#pragma unroll
+        for (int d = 0; d < D; ++d) mbar_init(bars + d, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+
+    // producer (lane 0): slice pass pt, row pair pj, source of the next unit, ring slot
     int pt = n_rp > 0 ? 0 : n_sl, pj = 0, pslot = 0;
-    int pactive = sl_lane == S - 1 ? L.last_active : 32;
     const unsigned char* psrc = codes + (size_t)sl_lane * kUnit2;
     auto issue = [&]() {
         if (pt < n_sl) {
-            if (lane < pactive) {
-                const unsigned char* src = psrc + lane * 16;
-                unsigned char* dst = ring_lane + pslot;
-                const int istride = pactive * 16;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) cp_async16(dst + i * 512, src + i * istride);
-                cp_async8(dst + 2048 - lane * 8, psrc + pactive * 64 + (lane >> 1) * 8);
+            if (lane == 0) {
+                const uint32_t bytes = (sl_lane + pt * Wc) == S - 1 ? (uint32_t)L.last_unit : (uint32_t)kUnit2;
+                mbar_expect_tx(bars + pslot, bytes);
+                bulk_copy_g2s(ring + pslot * kUnit2, psrc, bytes, bars + pslot);
             }
             psrc += rp_stride;
             if (++pj == n_rp) {
                 pj = 0;
                 ++pt;
-                const int sl = sl_lane + pt * Wc;
-                pactive = sl == S - 1 ? L.last_active : 32;
-                psrc = codes + (size_t)sl * kUnit2;
+                psrc = codes + (size_t)(sl_lane + pt * Wc) * kUnit2;
             }
         }
-        cp_async_commit();
-        pslot = pslot + kSlot == D * kSlot ? 0 : pslot + kSlot;
+        pslot = pslot + 1 == D ? 0 : pslot + 1;
     };
-    // One unit per warp goes out before anything else: the packed planes do not depend on earlier work of the
-    // stream (see ptqtp_gemv), x and y do.  Then wait for that earlier work, fetch x ahead of the rest of
-    // the weight stream (the whole CTA waits for x; its loads must not queue behind the stream), then fill
-    // the ring.
-    issue();
+    // The packed planes do not depend on earlier work of the stream (see ptqtp_gemv), x and y do: fill the ring,
+    // then wait for that work, then fetch x.
+#pragma unroll
+    for (int d = 0; d < D; ++d) issue();
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int xstep = blockDim.x * 8;
     const int xbase = (threadIdx.x & ~31) * 8, xlane = (threadIdx.x & 31) * 8;
@@ -189,9 +220,6 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
         xraw[p] = make_uint4(0u, 0u, 0u, 0u);
         if (base < L.k) xraw[p] = __ldg(reinterpret_cast<const uint4*>(x + base));
     }
-#pragma unroll
-    for (int d = 1; d < D; ++d) issue();
-
 #pragma unroll
     for (int p = 0; p < kPre; ++p) {
         if (xbase + p * xstep < L.k) {
@@ -208,6 +236,8 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     __syncthreads();
 
     int cslot = 0;
+    uint32_t phase = 0;                                 // parity of the ring pass being consumed
+    bool failed = false;
     for (int t = 0; t < n_sl; ++t) {
         const int sl = sl_lane + t * Wc;
         const int active = sl == S - 1 ? L.last_active : 32;
@@ -229,16 +259,27 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
         // the unmasked word stands for all four fields at once and starts at minus (1 + 4 + 16 + 64) times it
         const int n0 = -mt.y, n1 = -(mt.y << 2), n2 = -(mt.y << 4), n3 = -(mt.y * 85);
         float* ppart = partial + (size_t)wi * 2 * S + sl + (lane >> 4) * S;
+        // a slot holds the unit as it lies in memory: atom (i, l) at 16 (i A + l), the scale quads after the atoms
+        const int ln = live ? lane : 0;
+        const int atom_stride = active * 16;
+        const int scale_off = active * 64 + (ln >> 1) * 8 - ln * 16;
         for (int j = 0; j < n_rp; ++j) {
-            cp_async_wait<D - 1>();
-            const unsigned char* buf = ring_lane + cslot;
+            {   // wait (bounded) for the unit in slot cslot
+                uint64_t* bar = bars + cslot;
+                const int limit = failed ? kSpinLimitAfterFailure : kSpinLimit;
+                int spins = 0;
+                while (!mbar_try_wait(bar, phase)) {
+                    if (++spins >= limit) { failed = true; break; }
+                }
+            }
+            const unsigned char* buf = ring + cslot * kUnit2 + ln * 16;
             // Fields 0..2 are masked out of each code word; the unmasked word gives the sum of all four fields
             // (a byte is q0 + 4 q1 + 16 q2 + 64 q3 <= 170), so field 3 is "all" minus the other three.
             int ah[4] = {0, 0, 0, 0};
             int al[4] = {n0, n1, n2, n3};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint4 cw = *reinterpret_cast<const uint4*>(buf + i * 512);
+                const uint4 cw = *reinterpret_cast<const uint4*>(buf + i * atom_stride);
                 const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
                 for (int ww = 0; ww < 4; ++ww) {
@@ -252,27 +293,29 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                     al[3] = dot_uu(w[ww], xl[4 * i + ww], al[3]);
                 }
             }
-            const uint2 sc = *reinterpret_cast<const uint2*>(buf + 2048 - lane * 8);
+            const uint2 sc = *reinterpret_cast<const uint2*>(buf + scale_off);
             const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));   // alpha1, alpha2 of row 0
             const float2 s1 = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));   // ... of row 1
             // Q0..Q2 = 4^f * sum_j t_j X_j of fields 0..2; the unmasked word minus those three is field 3's
             const int Q0 = (ah[0] << 8) + al[0], Q1 = (ah[1] << 8) + al[1], Q2 = (ah[2] << 8) + al[2];
             const int Q3 = (ah[3] << 8) + al[3] - Q0 - Q1 - Q2;
-            // lanes past the slice's columns hold stale ring bytes and are zeroed explicitly
+            // lanes past the slice's columns redo lane 0 and are zeroed explicitly
             float y0 = live ? c0 * fmaf(0.25f, s0.y * (float)Q1, s0.x * (float)Q0) : 0.f;
             float y1 = live ? c1 * fmaf(0.25f, s1.y * (float)Q3, s1.x * (float)Q2) : 0.f;
+            // every lane has consumed the slot: lane 0 may refill it
+            __syncwarp();
             issue();
-            cslot = cslot + kSlot == D * kSlot ? 0 : cslot + kSlot;
+            if (++cslot == D) { cslot = 0; phase ^= 1u; }
             // lanes 0-15 reduce row 0, lanes 16-31 row 1
             const float send = (lane & 16) ? y0 : y1;
             float v = ((lane & 16) ? y1 : y0) + __shfl_xor_sync(0xffffffffu, send, 16);
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if ((lane & 15) == 0) *ppart = v;
+            if ((lane & 15) == 0) *ppart = failed ? __int_as_float(0x7fc00000) : v;
             ppart += (size_t)m * 2 * S;
         }
     }
-    cp_async_wait<0>();
+    if (failed && lane == 0) atomicExch(&g_gemv2_status, (int)PTQTP_ERR_CUDA);
     __syncthreads();
     const int rows = 2 * (rp1 - rp0);
     for (int r = threadIdx.x; r < rows; r += blockDim.x) {
@@ -284,9 +327,7 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
 }
 
 size_t smem_bytes(const Layout2& L, int rows_cap, int warps, int depth) {
-    const size_t nblk = (size_t)L.k / kLane2;
-    const size_t ring_off = (nblk * 136 + (size_t)rows_cap * L.slices * 4 + 15) / 16 * 16;
-    return ring_off + (size_t)warps * depth * kSlot;
+    return smem_layout2(L.k, L.slices, rows_cap, warps, depth).total;
 }
 
 template <int D>
@@ -320,6 +361,12 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
 
 }  // namespace
 
+ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st) {
+    cudaError_t e = cudaMemcpyFromSymbolAsync(status_host, g_gemv2_status, sizeof(int), 0, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+    return PTQTP_OK;
+}
+
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps, int depth,
                           cudaStream_t st) {
     const int S = L.slices;
@@ -336,7 +383,8 @@ ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* 
     const int rows_cap = 2 * ((L.nrp + grid - 1) / grid);
     const size_t budget = 227 * 1024;
     if (depth == 0) {
-        depth = 3;
+        // measured: two slots per warp are best when a CTA streams many units, three when it has few
+        depth = (long)((L.nrp + grid - 1) / grid) * S >= 64 ? 2 : 3;
         while (depth > 2 && smem_bytes(L, rows_cap, warps, depth) > budget) --depth;
     }
     const size_t smem = smem_bytes(L, rows_cap, warps, depth);

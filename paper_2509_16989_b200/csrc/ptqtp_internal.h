@@ -105,6 +105,7 @@ size_t skinny3_workspace_bytes(int k, int m);
 ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, void* workspace,
                             cudaStream_t st);
 ptqtp_status static_workspace_address(void** out);
+ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st);
 int sm_count();
 bool overlap_enabled();           // programmatic dependent launch of the GEMV kernels (ptqtp_set_overlap)
 

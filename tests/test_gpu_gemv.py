@@ -41,8 +41,12 @@ def test_format2_launch_configurations(warps, depth):
         c = make_case(N, K, seed=warps * 10 + depth)
         ref = oracle_y(c)
         packed = pack_case(c, binding.FORMAT_V2)
-        # shared memory: x as two byte planes + block records, the slice partials, warps * depth ring slots
-        smem = (K // 64) * 136 + 2 * -(-((N + 1) // 2) // 148) * -(-K // 2048) * 4 + 16 + warps * depth * 2304
+        # shared memory: x as two byte planes + block records, the slice partials, one mbarrier and one
+        # 2176-byte slot per ring entry
+        S = -(-K // 2048)
+        rows_cap = 2 * -(-((N + 1) // 2) // min(148, (N + 1) // 2))
+        bar_off = -(-((K // 64) * 136 + rows_cap * S * 4) // 8) * 8
+        smem = -(-(bar_off + warps * depth * 8) // 16) * 16 + warps * depth * 2176
         if smem > 227 * 1024:
             with pytest.raises(binding.PtqtpError) as e:
                 binding.ptqtp_gemv_cfg(packed, N, K, dev(c["x"]), k_split=warps, depth=depth, fmt=binding.FORMAT_V2)
@@ -382,3 +386,9 @@ def test_gemm_skinny_ws_argument_checks_and_exactness():
     with pytest.raises(binding.PtqtpError) as e:
         binding.ptqtp_gemm_skinny_ws(p1, N, K, dev(c["x"]), workspace=small, fmt=binding.FORMAT_V1)
     assert e.value.status == binding.ERR_CONFIG
+
+
+def test_kernel_status_is_healthy():
+    c = make_case(64, 4096, seed=60)
+    run_gemv(c, binding.FORMAT_V2)
+    assert binding.ptqtp_kernel_status() == 0
