@@ -36,7 +36,7 @@ UNIQUE_OF = {"q": "qo", "o": "qo", "k": "kv", "v": "kv", "gate": "gate_up", "up"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes in the ncu capture of the 14336x4096 launch of
 # the current GEMV kernel (profiles/gemv2_gate_up_14336x4096.md); set to None when the kernel changes
-DRAM_TRAFFIC_RATIO = 31234048.0 / 31232000.0
+DRAM_TRAFFIC_RATIO = 31232000.0 / 31232000.0
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -67,6 +67,23 @@ def dist_env():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     return rank, world, local
+
+
+# ----------------------------------------------------------------------------- replicas
+def max_over_ranks(ms, world, device=None):
+    """Slowest rank's time: the job is as fast as its slowest replica (no-op for one rank)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput_gbs(ms_per_step, world, step_bytes=None):
+    """Whole-job GB/s of `world` independent replicas that each move step_bytes per step (weak scaling)."""
+    return world * (STEP_BYTES if step_bytes is None else step_bytes) / (ms_per_step * 1e-3) / 1e9
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -306,14 +323,10 @@ def run_gpu(args):
     torch.cuda.synchronize()
     t_end = time.perf_counter()
     barrier()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), world, device)
     clocks = sampler.summary(t_begin, t_end)
     ms_per_step = ms / args.steps
-    value = world * STEP_BYTES / (ms_per_step * 1e-3) / 1e9
+    value = job_throughput_gbs(ms_per_step, world)
 
     # ---- parity spot check of what was just timed (sampled rows, fp64 oracle) ----
     parity = None
@@ -340,10 +353,30 @@ def run_gpu(args):
     xh = {m: torch.from_numpy(cases[UNIQUE_OF[m]]["x"].copy()).pin_memory() for m in MATRICES}
     yh = {m: torch.empty(LLAMA3_8B[m][0], dtype=torch.float16).pin_memory() for m in MATRICES}
 
-    def e2e_step(r):
+    def e2e_calls(r):
         for m in MATRICES:
             N, K = LLAMA3_8B[m]
             binding.ptqtp_gemv_host(sets[r][m], N, K, xh[m], yh[m], xs[m], ys[m], stream=stream)
+
+    # the host-buffer calls of a step are captured once per layer copy, like the device-resident steps
+    e2e_graphs = None
+    if not args.no_graph:
+        with torch.cuda.stream(stream):
+            e2e_calls(0)
+            stream.synchronize()
+            e2e_graphs = []
+            for r in range(R):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    e2e_calls(r)
+                e2e_graphs.append(g)
+
+    def e2e_step(r):
+        with torch.cuda.stream(stream):
+            if e2e_graphs is None:
+                e2e_calls(r)
+            else:
+                e2e_graphs[r].replay()
         stream.synchronize()
 
     for i in range(3):
@@ -355,12 +388,8 @@ def run_gpu(args):
         e2e_step(i % R)
     e1.record(stream)
     stream.synchronize()
-    e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * STEP_BYTES / (e2e_ms / e2e_steps * 1e-3) / 1e9
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, device)
+    e2e_value = job_throughput_gbs(e2e_ms / e2e_steps, world)
     h2d = sum(2 * LLAMA3_8B[m][1] for m in MATRICES)
     d2h = sum(2 * LLAMA3_8B[m][0] for m in MATRICES)
 
@@ -431,7 +460,9 @@ def run_gpu(args):
                      "kernel": "gemv2_kernel (7 launches per step; mean over the step)",
                      "bytes_per_launch_mean": STEP_BYTES / 7.0, "us_per_launch_mean": 1e3 * ms_per_step / 7.0},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "us_per_layer": 1e3 * e2e_ms / e2e_steps},
+                "steps": e2e_steps, "us_per_layer": 1e3 * e2e_ms / e2e_steps,
+                "launch": ("cuda graph of the 7 ptqtp_gemv_host calls" if e2e_graphs else "plain calls")
+                          + ", one stream synchronisation per step"},
         "gpu_launches": launches, "clocks": clocks, "parity": parity, "shapes": detail,
     }
     if world == 1 and not args.no_cpu:
