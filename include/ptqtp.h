@@ -218,14 +218,18 @@ PTQTP_API int ptqtp_last_cuda_error(void);
  * This call enqueues a copy of that word (0 = healthy) to *status_host on `stream`; read it after syncing. */
 PTQTP_API ptqtp_status ptqtp_kernel_status(int32_t *status_host /* host */, void *stream);
 
-/* Overlap of consecutive GEMV calls on one stream (process-wide switch, on by default; returns the old
- * value).  When on, format-2 GEMV kernels are launched with programmatic stream serialization: a call may
- * begin reading its `packed` blob while the GEMV call directly before it on the stream is still draining;
- * x is read and y written only after all earlier work on the stream has completed, so stream order holds
- * for them.  Consequence for the caller: the packed blob of a call must not be the output buffer of the
- * GEMV call directly before it.  Work of any other kind before a call is always complete before the call
- * reads anything.  Works inside CUDA graph capture. */
-PTQTP_API int ptqtp_set_overlap(int enabled);
+/* Overlap of consecutive GEMV calls on one stream (process-wide level, default 2; returns the old level).
+ * Level 0: plain launches.  Level 1: format-2 GEMV kernels are launched with programmatic stream
+ * serialization: a call may begin reading its `packed` blob while the GEMV call directly before it on the
+ * stream is still draining; x is used and y written only after all earlier work on the stream has completed,
+ * so stream order holds for them.  Consequence for the caller: the packed blob of a call must not be the
+ * output buffer of the GEMV call directly before it.  Work of any other kind before a call is always complete
+ * before the call reads anything.  Works inside CUDA graph capture.
+ * Level 2 adds a speculative read of x: the kernel also reads and converts x before earlier work has
+ * completed, reads it again afterwards and, if a single bit differs anywhere, converts it again from the
+ * second read; results are identical to level 1 in every case.  It pays when x was finished well before the
+ * call (k and v after q, up after gate share their x) and costs one comparison when it was not. */
+PTQTP_API int ptqtp_set_overlap(int level);
 
 /* Library version: major*10000 + minor*100 + patch. */
 PTQTP_API int ptqtp_version(void);

@@ -251,9 +251,12 @@ def ptqtp_kernel_status(stream=None):
     return int(out.value)
 
 
-def ptqtp_set_overlap(enabled):
-    """Switch the overlap of consecutive GEMV calls (programmatic dependent launch); returns the old setting."""
-    return bool(lib().ptqtp_set_overlap(1 if enabled else 0))
+def ptqtp_set_overlap(level):
+    """Overlap level of consecutive GEMV calls: 0 off, 1 programmatic dependent launch, 2 (default) also the
+    speculative read of x.  True/False mean 2/0.  Returns the old level."""
+    if level is True:
+        level = 2
+    return int(lib().ptqtp_set_overlap(int(level)))
 
 
 def ptqtp_parse_header(header_bytes):

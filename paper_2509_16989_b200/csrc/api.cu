@@ -5,9 +5,10 @@
 namespace ptqtp {
 
 static thread_local int g_last_cuda_error = 0;
-static int g_overlap = 1;
+static int g_overlap = 2;
 
 bool overlap_enabled() { return g_overlap != 0; }
+bool speculation_enabled() { return g_overlap >= 2; }
 
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
 
@@ -231,7 +232,7 @@ ptqtp_status ptqtp_kernel_status(int32_t* status_host, void* stream) {
 
 int ptqtp_set_overlap(int enabled) {
     const int old = g_overlap;
-    g_overlap = enabled ? 1 : 0;
+    g_overlap = enabled <= 0 ? 0 : enabled >= 2 ? 2 : 1;
     return old;
 }
 

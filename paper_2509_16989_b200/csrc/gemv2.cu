@@ -150,7 +150,7 @@ __host__ __device__ inline Smem2 smem_layout2(int k, int slices, int rows_cap, i
 template <int D>
 __global__ void __launch_bounds__(kMaxThreads2, 1)
 gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
-             __half* __restrict__ y, int rows_cap, int rp_base, int rp_rem) {
+             __half* __restrict__ y, int rows_cap, int rp_base, int rp_rem, int speculate) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int nblk = L.k / kLane2;
     uint32_t* xhi = reinterpret_cast<uint32_t*>(smem);
@@ -210,30 +210,55 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     // then wait for that work, then fetch x.
 #pragma unroll
     for (int d = 0; d < D; ++d) issue();
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Activations.  Earlier work of the stream may still be writing x, so x counts only after the wait below.
+    // But most calls of a decoder read an x that was finished long before (k and v after q, up after gate): x
+    // is therefore read and converted speculatively now, while the previous kernel drains, and read again
+    // after the wait; if any thread of the CTA sees a difference, everything is converted again from the
+    // second read.  Both reads go to L2 (ld.global.cg), the point of coherence, never through L1.
     const int xstep = blockDim.x * 8;
     const int xbase = (threadIdx.x & ~31) * 8, xlane = (threadIdx.x & 31) * 8;
     uint4 xraw[kPre];
+    if (speculate) {
+#pragma unroll
+        for (int p = 0; p < kPre; ++p) {
+            const int base = xbase + p * xstep + xlane;
+            xraw[p] = make_uint4(0u, 0u, 0u, 0u);
+            if (base < L.k) xraw[p] = __ldcg(reinterpret_cast<const uint4*>(x + base));
+        }
+#pragma unroll
+        for (int p = 0; p < kPre; ++p) {
+            if (xbase + p * xstep < L.k) {
+                const int base = xbase + p * xstep + xlane;
+                convert_x8(xraw[p], base, base < L.k, xhi, xlo, meta);
+            }
+        }
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    int stale = speculate ? 0 : 1;
 #pragma unroll
     for (int p = 0; p < kPre; ++p) {
         const int base = xbase + p * xstep + xlane;
-        xraw[p] = make_uint4(0u, 0u, 0u, 0u);
-        if (base < L.k) xraw[p] = __ldg(reinterpret_cast<const uint4*>(x + base));
+        uint4 now = make_uint4(0u, 0u, 0u, 0u);
+        if (base < L.k) now = __ldcg(reinterpret_cast<const uint4*>(x + base));
+        if (speculate) stale |= (now.x != xraw[p].x) | (now.y != xraw[p].y) | (now.z != xraw[p].z) | (now.w != xraw[p].w);
+        xraw[p] = now;
     }
-#pragma unroll
-    for (int p = 0; p < kPre; ++p) {
-        if (xbase + p * xstep < L.k) {
-            const int base = xbase + p * xstep + xlane;
-            convert_x8(xraw[p], base, base < L.k, xhi, xlo, meta);
-        }
-    }
-    for (int wb = xbase + kPre * xstep; wb < L.k; wb += xstep) {       // very long K: the rest, loaded late
+    for (int wb = xbase + kPre * xstep; wb < L.k; wb += xstep) {       // very long K: the rest is never speculated
         const int base = wb + xlane;
         uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-        if (base < L.k) raw = __ldg(reinterpret_cast<const uint4*>(x + base));
+        if (base < L.k) raw = __ldcg(reinterpret_cast<const uint4*>(x + base));
         convert_x8(raw, base, base < L.k, xhi, xlo, meta);
     }
-    __syncthreads();
+    if (__syncthreads_or(stale)) {                       // also publishes the converted x when nothing was stale
+#pragma unroll
+        for (int p = 0; p < kPre; ++p) {
+            if (xbase + p * xstep < L.k) {
+                const int base = xbase + p * xstep + xlane;
+                convert_x8(xraw[p], base, base < L.k, xhi, xlo, meta);
+            }
+        }
+        __syncthreads();
+    }
 
     int cslot = 0;
     uint32_t phase = 0;                                 // parity of the ring pass being consumed
@@ -354,7 +379,7 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
     cfg.numAttrs = overlap_enabled() ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, L, static_cast<const unsigned char*>(packed),
                                        reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap,
-                                       L.nrp / grid, L.nrp % grid);
+                                       L.nrp / grid, L.nrp % grid, speculation_enabled() ? 1 : 0);
     if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
     return PTQTP_OK;
 }

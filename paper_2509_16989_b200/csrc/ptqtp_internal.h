@@ -107,6 +107,7 @@ ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const u
 ptqtp_status static_workspace_address(void** out);
 ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st);
 int sm_count();
+bool speculation_enabled();       // speculative read of x before the dependency wait (ptqtp_set_overlap(2))
 bool overlap_enabled();           // programmatic dependent launch of the GEMV kernels (ptqtp_set_overlap)
 
 }  // namespace ptqtp

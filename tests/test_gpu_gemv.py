@@ -292,8 +292,9 @@ def test_decomposed_weights_end_to_end():
     assert rel < 2.5 * err
 
 
+@pytest.mark.parametrize("level", [1, 2])
 @pytest.mark.parametrize("graph", [False, True])
-def test_overlapped_chain_keeps_stream_order(graph):
+def test_overlapped_chain_keeps_stream_order(graph, level):
     # y1 = layer1(x), y2 = layer2(y1), y3 = layer1(y2): each call's x is the previous call's y, so a call
     # that read x before its predecessor finished would be caught.  Checked link by link against the oracle.
     N = K = 2048
@@ -303,7 +304,7 @@ def test_overlapped_chain_keeps_stream_order(graph):
     p1, p2 = pack_case(c1, binding.FORMAT_V2), pack_case(c2, binding.FORMAT_V2)
     x = dev(c1["x"])
     ys = [torch.empty(N, dtype=torch.float16, device="cuda") for _ in range(3)]
-    assert binding.ptqtp_set_overlap(True) in (True, False)
+    assert binding.ptqtp_set_overlap(level) in (0, 1, 2)
 
     def chain():
         binding.ptqtp_gemv(p1, N, K, x, y=ys[0], fmt=binding.FORMAT_V2)
@@ -333,7 +334,7 @@ def test_overlapped_chain_keeps_stream_order(graph):
         ref = oracle_y(dict(cc, x=xin))
         assert_parity(yout, ref, xin, what)
     # and with the overlap switched off the results are bit-identical
-    assert binding.ptqtp_set_overlap(False) is True
+    assert binding.ptqtp_set_overlap(0) == level
     try:
         with torch.cuda.stream(stream):
             chain()
@@ -341,7 +342,39 @@ def test_overlapped_chain_keeps_stream_order(graph):
         for y, ref in zip(ys, h):
             assert np.array_equal(y.cpu().numpy().view(np.uint16), ref.view(np.uint16))
     finally:
-        binding.ptqtp_set_overlap(True)
+        binding.ptqtp_set_overlap(2)
+
+
+def test_speculative_read_sees_activations_written_just_before():
+    # x is rewritten on the stream (by a copy, by an elementwise kernel) directly before each call, alternating
+    # between two vectors that differ in one element only; every call must use the value written last.
+    N, K = 512, 4096
+    c = make_case(N, K, seed=60)
+    packed = pack_case(c, binding.FORMAT_V2)
+    xa = c["x"].copy()
+    xb = c["x"].copy()
+    xb[K - 3] = np.float16(-float(xb[K - 3]) + 0.25)
+    da, db = dev(xa), dev(xb)
+    x = torch.empty(K, dtype=torch.float16, device="cuda")
+    ys = [torch.empty(N, dtype=torch.float16, device="cuda") for _ in range(6)]
+    assert binding.ptqtp_set_overlap(2) in (0, 1, 2)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i, y in enumerate(ys):
+            src = da if i % 2 == 0 else db
+            if i % 3 == 0:
+                x.copy_(src)
+            else:
+                torch.add(src, 0, out=x)
+            binding.ptqtp_gemv(packed, N, K, x, y=y, fmt=binding.FORMAT_V2)
+        stream.synchronize()
+    ra, rb = oracle_y(dict(c, x=xa)), oracle_y(dict(c, x=xb))
+    assert not np.array_equal(ra.astype(np.float16), rb.astype(np.float16))
+    for i, y in enumerate(ys):
+        assert_parity(y.cpu().numpy(), ra if i % 2 == 0 else rb, xa if i % 2 == 0 else xb, "call %d" % i)
+    assert np.array_equal(ys[0].cpu().numpy().view(np.uint16), ys[2].cpu().numpy().view(np.uint16))
+    assert np.array_equal(ys[1].cpu().numpy().view(np.uint16), ys[3].cpu().numpy().view(np.uint16))
+    assert not np.array_equal(ys[0].cpu().numpy().view(np.uint16), ys[1].cpu().numpy().view(np.uint16))
 
 
 @pytest.mark.parametrize("N,K,M", [(1, 128, 1), (5, 256, 3), (7, 1152, 4), (33, 2048, 5), (130, 3200, 8), (257, 5120, 12),
