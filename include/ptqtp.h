@@ -138,10 +138,11 @@ PTQTP_API ptqtp_status ptqtp_gemv(const ptqtp_shape *shape /* host */, const voi
 
 /* Small-batch variant: Y[m,:] = layer(X[m,:]) for m < M, 1 <= M <= PTQTP_MAX_BATCH.
  * X: device fp16 [M*K] row-major; Y: device fp16 [M*N] row-major.  Same definition per row of X.
- * Format 2, M >= 2: the planes are decoded once per pass of up to 8 batch rows (fewer when K is long: the
- * activations of a pass live in shared memory) and contracted on the tensor cores with int8 warp MMAs against
- * 15-bit block-fixed-point activations (blocks of 128 columns), exact int32 sums, fp32 scale epilogue.
- * M = 1 runs the batch-1 kernel.  Format 1: one batch-1 pass per row. */
+ * Format 2, M >= 2: the planes are contracted on the tensor cores with int8 warp MMAs against 15-bit
+ * block-fixed-point activations (blocks of 128 columns), exact int32 sums, fp32 scale epilogue.  M = 2..4 take
+ * one pass over the planes at about the cost of a batch-1 call (the activations stay in registers); larger M
+ * decode the planes once per pass of up to 8 batch rows (fewer when K is long: the activations of a pass live
+ * in shared memory).  M = 1 runs the batch-1 kernel.  Format 1: one batch-1 pass per row. */
 PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, const void *packed,
                                size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                void *stream);
@@ -195,9 +196,13 @@ PTQTP_API ptqtp_status ptqtp_gemv_host(const ptqtp_shape *shape /* host */, cons
  * arith: accumulation of the sign-selected activations -- 0 = fp32 accumulator fed by mixed-precision
  * FMAs (fp16 operands), 1 = fp16x2 chains of 4 flushed into fp32, 2 = chains of 8, -1 = library choice.
  * PTQTP_ERR_CONFIG if the combination is not built.
- * For a format-2 blob the arguments mean: rows_per_warp must be 0; k_split = warps per CTA (1..16, 0 = auto);
- * ctas_per_sm must be 0 or 1 (one persistent CTA per SM); depth = slice units in flight per warp
- * (2, 3, 4, 6, 8; 0 = auto); arith must be -1 or 3 (integer dot products). */
+ * For a format-2 blob the arguments mean: rows_per_warp must be 0; arith = -1 (library choice), 3 (masks and
+ * integer dot products on the CUDA cores) or 4 (int8 tensor-core MMAs, the kernel behind ptqtp_gemm_skinny for
+ * two to four rows).  arith 3: k_split = warps per CTA (1..16 / ctas_per_sm, 0 = auto: 4 to 8, so that the CTAs
+ * of several consecutive launches fit on an SM together; 16 serves a call that runs alone best);
+ * ctas_per_sm = CTAs of this launch per SM (1..4, 0 = 1); depth = slice units in flight per warp (2, 3, 4, 6,
+ * 8; 0 = 2).  arith 4: k_split = warps per CTA (4, 8 or 16, 0 = auto); ctas_per_sm 1 or 2 (0 = 1); depth =
+ * stages (four slice units each) per team of four warps (2..8, 0 = auto). */
 PTQTP_API ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                             const uint16_t *x, uint16_t *y, int32_t rows_per_warp, int32_t k_split,
                             int32_t ctas_per_sm, int32_t depth, int32_t arith, void *stream);
@@ -212,8 +217,9 @@ PTQTP_API const char *ptqtp_status_string(ptqtp_status status);
 /* The cudaError_t (as int) behind the calling thread's most recent PTQTP_ERR_CUDA, else 0. */
 PTQTP_API int ptqtp_last_cuda_error(void);
 
-/* Device-side health of the batch-1 kernel on the current device.  The format-2 GEMV streams the packed planes
- * with bulk copies and waits for each with a bounded number of polls; if a wait ever gives up, the kernel
+/* Device-side health of the format-2 kernels that stream the packed planes with bulk copies (batch 1, and the
+ * small-batch kernel for two to four rows) on the current device.  They wait for each copy with a bounded
+ * number of polls; if a wait ever gives up, the kernel
  * writes NaN to the rows it could not finish, records PTQTP_ERR_CUDA in a device word and still terminates.
  * This call enqueues a copy of that word (0 = healthy) to *status_host on `stream`; read it after syncing. */
 PTQTP_API ptqtp_status ptqtp_kernel_status(int32_t *status_host /* host */, void *stream);
@@ -225,10 +231,13 @@ PTQTP_API ptqtp_status ptqtp_kernel_status(int32_t *status_host /* host */, void
  * so stream order holds for them.  Consequence for the caller: the packed blob of a call must not be the
  * output buffer of the GEMV call directly before it.  Work of any other kind before a call is always complete
  * before the call reads anything.  Works inside CUDA graph capture.
- * Level 2 adds a speculative read of x: the kernel also reads and converts x before earlier work has
- * completed, reads it again afterwards and, if a single bit differs anywhere, converts it again from the
- * second read; results are identical to level 1 in every case.  It pays when x was finished well before the
- * call (k and v after q, up after gate share their x) and costs one comparison when it was not. */
+ * Level 2 adds speculative execution: the kernel reads x at once and computes everything into shared memory
+ * while earlier work of the stream may still be running, then waits for that work, reads x again and compares
+ * it bit by bit with its first read; y is written only after that, and if a single bit of x differed the whole
+ * computation is repeated from the second read.  Results are identical to level 1 in every case.  It pays when
+ * x was finished before the call directly ahead of this one started (k and v after q, up after gate, any call
+ * behind work that is not a GEMV of this library) and costs a second pass over the matrix when it was not (y of
+ * the GEMV directly ahead used as x). */
 PTQTP_API int ptqtp_set_overlap(int level);
 
 /* Library version: major*10000 + minor*100 + patch. */

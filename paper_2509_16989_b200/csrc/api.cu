@@ -52,11 +52,22 @@ static ptqtp_status check_packed(const ptqtp_shape* shape, const void* packed, s
     return PTQTP_OK;
 }
 
+static int default_gemv_arith() { return 3; }
+
 static ptqtp_status gemv_any(const AnyLayout& L, const void* packed, const uint16_t* x, uint16_t* y, int p0, int p1,
                              int p2, int p3, int p4, cudaStream_t st) {
     if (L.v2) {
-        if (p0 != 0 || p2 > 1 || (p4 != -1 && p4 != 3)) return PTQTP_ERR_CONFIG;
-        return launch_gemv2(L.l2, packed, x, y, p1, p3, st);
+        if (p0 != 0 || (p4 != -1 && p4 != 3 && p4 != 4)) return PTQTP_ERR_CONFIG;
+        if (p4 == 4) {                       // tensor-core kernel
+            const ptqtp_status s = launch_gemv3(L.l2, packed, 1, x, y, p1, p2, p3, st);
+            return s == PTQTP_ERR_SHAPE ? PTQTP_ERR_CONFIG : s;
+        }
+        if (p2 > 4) return PTQTP_ERR_CONFIG;
+        if (p4 == -1 && p1 == 0 && p2 == 0 && p3 == 0 && default_gemv_arith() == 4) {
+            const ptqtp_status s = launch_gemv3(L.l2, packed, 1, x, y, 0, 0, 0, st);
+            if (s != PTQTP_ERR_SHAPE) return s;          // very long K: the CUDA-core kernel takes it
+        }
+        return launch_gemv2(L.l2, packed, x, y, p1, p2, p3, st);
     }
     return launch_gemv(L.l1, packed, x, y, p0, p1, p2, p3, p4, st);
 }
@@ -126,8 +137,14 @@ ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, siz
     if (m < 1 || m > PTQTP_MAX_BATCH) return PTQTP_ERR_SHAPE;
     if (!aligned16(X) || !aligned16(Y)) return PTQTP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // format 2: one batch row is fastest on the batch-1 kernel (measured); two or more go to the tensor-core kernel
-    if (L.v2) return m == 1 ? launch_gemv2(L.l2, packed, X, Y, 0, 0, st) : launch_skinny2(L.l2, packed, m, X, Y, st);
+    if (L.v2) {
+        // two to four rows cost the same as one on the register-stationary tensor-core kernel
+        if (m >= 2 && m <= 4) {
+            const ptqtp_status s4 = launch_gemv3(L.l2, packed, m, X, Y, 0, 0, 0, st);
+            if (s4 != PTQTP_ERR_SHAPE) return s4;
+        }
+        return m == 1 ? launch_gemv2(L.l2, packed, X, Y, 0, 0, 0, st) : launch_skinny2(L.l2, packed, m, X, Y, st);
+    }
     return launch_gemm_skinny(L.l1, packed, m, X, Y, st);
 }
 

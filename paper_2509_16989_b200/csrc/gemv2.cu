@@ -24,12 +24,20 @@
 //     device status word (ptqtp_kernel_status) and still runs to the end.
 //   * Rows are reduced over the lanes by shuffles, over the slices through shared memory in a fixed order
 //     (deterministic), rounded once to fp16.
+//   * Two CTAs per SM whenever the activations leave room: the head and the tail of one CTA (fetching x, the
+//     final reduction) overlap the streaming of the other, also across consecutive launches.
+//   * Speculative execution under programmatic dependent launch.  x and y belong to the stream's order, the
+//     packed planes do not.  Earlier work of the stream may still be running when this kernel starts; most
+//     calls of a decoder read an x that was finished long before.  The kernel therefore reads x at once,
+//     computes everything into shared memory, then waits for the earlier work, reads x again and compares it
+//     bit by bit with its first read (kept in shared memory).  Only then y is written; if a single bit of x
+//     differed, the whole computation is repeated from the second read.  Results never depend on the timing.
 #include <cuda_fp16.h>
 #include "ptqtp_internal.h"
 
 namespace ptqtp {
 
-// Device-side status of the GEMV kernel: set when a bounded wait for a bulk copy gave up.
+// Device-side status of the GEMV kernels: set when a bounded wait for a bulk copy gave up.
 __device__ int g_gemv2_status = 0;
 
 namespace {
@@ -77,7 +85,7 @@ __device__ __forceinline__ int dot_uu(uint32_t a, uint32_t x, int c) {
 //   xhi, xlo : [K/64 blocks][16 words]  bytes of hi_j / lo_j in column order
 //   meta     : [K/64 blocks] (2^-s as float bits, sum_j X_j)
 // Eight adjacent threads share a 64-column block (8 columns each); the whole warp must call this.
-__device__ __forceinline__ void convert_x8(uint4 raw, int base, bool valid, uint32_t* xhi, uint32_t* xlo, int2* meta) {
+__device__ __noinline__ void convert_x8(uint4 raw, int base, bool valid, uint32_t* xhi, uint32_t* xlo, int2* meta) {
     const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
     // block maximum of |x| on the fp16 bit patterns (ordered like the values once the sign is cleared)
     const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -131,16 +139,16 @@ __device__ __forceinline__ void convert_x8(uint4 raw, int base, bool valid, uint
     }
 }
 
-constexpr int kPre = 4;                    // x loads per thread issued ahead of the weight stream
-
-// Shared memory: x as two byte planes and block records, the per-slice partial sums, one mbarrier per ring slot,
-// then the ring (one slice unit, kUnit2 bytes, per slot; D slots per warp).
+// Shared memory: x as two byte planes and block records, the first read of x (fp16 as read, only when executing
+// speculatively), the per-slice partial sums, one mbarrier per ring slot, then the ring (one slice unit, kUnit2
+// bytes, per slot; D slots per warp).
 struct Smem2 {
-    size_t partial_off, bar_off, ring_off, total;
+    size_t raw_off, partial_off, bar_off, ring_off, total;
 };
-__host__ __device__ inline Smem2 smem_layout2(int k, int slices, int rows_cap, int warps, int depth) {
+__host__ __device__ inline Smem2 smem_layout2(int k, int slices, int rows_cap, int warps, int depth, int speculate) {
     Smem2 m;
-    m.partial_off = (size_t)(k / kLane2) * 136;
+    m.raw_off = ((size_t)(k / kLane2) * 136 + 15) / 16 * 16;
+    m.partial_off = m.raw_off + (speculate ? (size_t)2 * k : 0);
     m.bar_off = (m.partial_off + (size_t)rows_cap * slices * 4 + 7) / 8 * 8;
     m.ring_off = (m.bar_off + (size_t)warps * depth * 8 + 15) / 16 * 16;
     m.total = m.ring_off + (size_t)warps * depth * kUnit2;
@@ -157,13 +165,14 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     uint32_t* xlo = xhi + nblk * 16;
     int2* meta = reinterpret_cast<int2*>(xlo + nblk * 16);
     const int warps = blockDim.x >> 5;
-    const Smem2 sm = smem_layout2(L.k, L.slices, rows_cap, warps, D);
+    const Smem2 sm = smem_layout2(L.k, L.slices, rows_cap, warps, D, speculate);
+    uint4* first_read = reinterpret_cast<uint4*>(smem + sm.raw_off);        // x as read before the dependency wait
     float* partial = reinterpret_cast<float*>(smem + sm.partial_off);       // [rows_cap][slices]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bar_off) + warp * D;
     unsigned char* ring = smem + sm.ring_off + (size_t)warp * D * kUnit2;
 
-    // Let the next kernel on the stream start its own weight prefetch while this one drains.
+    // Let the next kernel on the stream start while this one runs.
     asm volatile("griddepcontrol.launch_dependents;");
 
     // this CTA's row pairs, and this warp's share of their slice units
@@ -179,6 +188,7 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     const int n_rp = idle ? 0 : max(0, (rp1 - rp0 - wi + m - 1) / m);
     const unsigned char* codes = packed + L.codes_off + (size_t)(rp0 + wi) * L.strip;
     const size_t rp_stride = (size_t)m * L.strip;
+    const int nchunks = L.k >> 3, cthreads = blockDim.x;
 
     if (lane == 0) {
 #pragma unroll
@@ -188,8 +198,8 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     __syncwarp();
 
     // producer (lane 0): slice pass pt, row pair pj, source of the next unit, ring slot
-    int pt = n_rp > 0 ? 0 : n_sl, pj = 0, pslot = 0;
-    const unsigned char* psrc = codes + (size_t)sl_lane * kUnit2;
+    int pt = 0, pj = 0, pslot = 0;
+    const unsigned char* psrc = codes;
     auto issue = [&]() {
         if (pt < n_sl) {
             if (lane == 0) {
@@ -206,139 +216,142 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
         }
         pslot = pslot + 1 == D ? 0 : pslot + 1;
     };
-    // The packed planes do not depend on earlier work of the stream (see ptqtp_gemv), x and y do: fill the ring,
-    // then wait for that work, then fetch x.
-#pragma unroll
-    for (int d = 0; d < D; ++d) issue();
-    // Activations.  Earlier work of the stream may still be writing x, so x counts only after the wait below.
-    // But most calls of a decoder read an x that was finished long before (k and v after q, up after gate): x
-    // is therefore read and converted speculatively now, while the previous kernel drains, and read again
-    // after the wait; if any thread of the CTA sees a difference, everything is converted again from the
-    // second read.  Both reads go to L2 (ld.global.cg), the point of coherence, never through L1.
-    const int xstep = blockDim.x * 8;
-    const int xbase = (threadIdx.x & ~31) * 8, xlane = (threadIdx.x & 31) * 8;
-    uint4 xraw[kPre];
-    if (speculate) {
-#pragma unroll
-        for (int p = 0; p < kPre; ++p) {
-            const int base = xbase + p * xstep + xlane;
-            xraw[p] = make_uint4(0u, 0u, 0u, 0u);
-            if (base < L.k) xraw[p] = __ldcg(reinterpret_cast<const uint4*>(x + base));
-        }
-#pragma unroll
-        for (int p = 0; p < kPre; ++p) {
-            if (xbase + p * xstep < L.k) {
-                const int base = xbase + p * xstep + xlane;
-                convert_x8(xraw[p], base, base < L.k, xhi, xlo, meta);
-            }
-        }
-    }
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    int stale = speculate ? 0 : 1;
-#pragma unroll
-    for (int p = 0; p < kPre; ++p) {
-        const int base = xbase + p * xstep + xlane;
-        uint4 now = make_uint4(0u, 0u, 0u, 0u);
-        if (base < L.k) now = __ldcg(reinterpret_cast<const uint4*>(x + base));
-        if (speculate) stale |= (now.x != xraw[p].x) | (now.y != xraw[p].y) | (now.z != xraw[p].z) | (now.w != xraw[p].w);
-        xraw[p] = now;
-    }
-    for (int wb = xbase + kPre * xstep; wb < L.k; wb += xstep) {       // very long K: the rest is never speculated
-        const int base = wb + xlane;
-        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-        if (base < L.k) raw = __ldcg(reinterpret_cast<const uint4*>(x + base));
-        convert_x8(raw, base, base < L.k, xhi, xlo, meta);
-    }
-    if (__syncthreads_or(stale)) {                       // also publishes the converted x when nothing was stale
-#pragma unroll
-        for (int p = 0; p < kPre; ++p) {
-            if (xbase + p * xstep < L.k) {
-                const int base = xbase + p * xstep + xlane;
-                convert_x8(xraw[p], base, base < L.k, xhi, xlo, meta);
-            }
-        }
-        __syncthreads();
-    }
 
     int cslot = 0;
     uint32_t phase = 0;                                 // parity of the ring pass being consumed
-    bool failed = false;
-    for (int t = 0; t < n_sl; ++t) {
-        const int sl = sl_lane + t * Wc;
-        const int active = sl == S - 1 ? L.last_active : 32;
-        const bool live = lane < active;
-        // this lane's X block for the slice stays in registers
-        uint32_t xh[16], xl[16];
-        const int blk = sl * 32 + (live ? lane : 0);
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            const int pos = blk * 16 + ((v ^ ((blk >> 1) & 3)) << 2);
-            const uint4 a = *reinterpret_cast<const uint4*>(xhi + pos);
-            const uint4 b = *reinterpret_cast<const uint4*>(xlo + pos);
-            xh[4 * v] = a.x; xh[4 * v + 1] = a.y; xh[4 * v + 2] = a.z; xh[4 * v + 3] = a.w;
-            xl[4 * v] = b.x; xl[4 * v + 1] = b.y; xl[4 * v + 2] = b.z; xl[4 * v + 3] = b.w;
+    bool failed = false, waited = false;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        // Pass 0 is speculative when allowed: x is read before earlier work of the stream is known to be complete.
+        const bool spec = speculate && attempt == 0;
+        if (!spec && !waited) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            waited = true;
         }
-        const int2 mt = meta[blk];
-        const float c0 = live ? __int_as_float(mt.x) : 0.f, c1 = 0.0625f * c0;
-        // sum_j t_j X_j = sum_j q_j X_j - sum_j X_j: the low accumulators start at minus 4^f times the block sum;
-        // the unmasked word stands for all four fields at once and starts at minus (1 + 4 + 16 + 64) times it
-        const int n0 = -mt.y, n1 = -(mt.y << 2), n2 = -(mt.y << 4), n3 = -(mt.y * 85);
-        float* ppart = partial + (size_t)wi * 2 * S + sl + (lane >> 4) * S;
-        // a slot holds the unit as it lies in memory: atom (i, l) at 16 (i A + l), the scale quads after the atoms
-        const int ln = live ? lane : 0;
-        const int atom_stride = active * 16;
-        const int scale_off = active * 64 + (ln >> 1) * 8 - ln * 16;
-        for (int j = 0; j < n_rp; ++j) {
-            {   // wait (bounded) for the unit in slot cslot
-                uint64_t* bar = bars + cslot;
-                const int limit = failed ? kSpinLimitAfterFailure : kSpinLimit;
-                int spins = 0;
-                while (!mbar_try_wait(bar, phase)) {
-                    if (++spins >= limit) { failed = true; break; }
+        pt = n_rp > 0 ? 0 : n_sl;
+        pj = 0;
+        psrc = codes + (size_t)sl_lane * kUnit2;
+        // x -> block fixed point in shared memory, four 8-column chunks per thread in flight.  Reads go to L2
+        // (ld.global.cg), the point of coherence, never through L1.  The first reads are issued before the ring
+        // is filled (behind the fill they would wait for all of it); the packed planes do not depend on earlier
+        // work of the stream, so the fill never waits for that work.
+        bool filled = false;
+        for (int cb = (int)threadIdx.x; (cb & ~31) < nchunks; cb += 4 * cthreads) {
+            uint4 r[4];
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                const int c = cb + p * cthreads;
+                r[p] = make_uint4(0u, 0u, 0u, 0u);
+                if (c < nchunks) r[p] = __ldcg(reinterpret_cast<const uint4*>(x) + c);
+            }
+            if (!filled) {
+                filled = true;
+#pragma unroll
+                for (int d = 0; d < D; ++d) issue();
+            }
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                const int c = cb + p * cthreads;
+                if ((c & ~31) < nchunks) {
+                    if (spec && c < nchunks) first_read[c] = r[p];
+                    convert_x8(r[p], c << 3, c < nchunks, xhi, xlo, meta);
                 }
             }
-            const unsigned char* buf = ring + cslot * kUnit2 + ln * 16;
-            // Fields 0..2 are masked out of each code word; the unmasked word gives the sum of all four fields
-            // (a byte is q0 + 4 q1 + 16 q2 + 64 q3 <= 170), so field 3 is "all" minus the other three.
-            int ah[4] = {0, 0, 0, 0};
-            int al[4] = {n0, n1, n2, n3};
+        }
+        if (!filled) {                                  // a warp with no part of x to convert
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint4 cw = *reinterpret_cast<const uint4*>(buf + i * atom_stride);
-                const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
+            for (int d = 0; d < D; ++d) issue();
+        }
+        __syncthreads();
+
+        for (int t = 0; t < n_sl; ++t) {
+            const int sl = sl_lane + t * Wc;
+            const int active = sl == S - 1 ? L.last_active : 32;
+            const bool live = lane < active;
+            // this lane's X block for the slice stays in registers
+            uint32_t xh[16], xl[16];
+            const int blk = sl * 32 + (live ? lane : 0);
 #pragma unroll
-                for (int ww = 0; ww < 4; ++ww) {
-#pragma unroll
-                    for (int f = 0; f < 3; ++f) {
-                        const uint32_t mk = w[ww] & (0x03030303u << (2 * f));
-                        ah[f] = dot_us(mk, xh[4 * i + ww], ah[f]);
-                        al[f] = dot_uu(mk, xl[4 * i + ww], al[f]);
+            for (int v = 0; v < 4; ++v) {
+                const int pos = blk * 16 + ((v ^ ((blk >> 1) & 3)) << 2);
+                const uint4 a = *reinterpret_cast<const uint4*>(xhi + pos);
+                const uint4 b = *reinterpret_cast<const uint4*>(xlo + pos);
+                xh[4 * v] = a.x; xh[4 * v + 1] = a.y; xh[4 * v + 2] = a.z; xh[4 * v + 3] = a.w;
+                xl[4 * v] = b.x; xl[4 * v + 1] = b.y; xl[4 * v + 2] = b.z; xl[4 * v + 3] = b.w;
+            }
+            const int2 mt = meta[blk];
+            const float c0 = live ? __int_as_float(mt.x) : 0.f, c1 = 0.0625f * c0;
+            // sum_j t_j X_j = sum_j q_j X_j - sum_j X_j: the low accumulators start at minus 4^f times the block sum;
+            // the unmasked word stands for all four fields at once and starts at minus (1 + 4 + 16 + 64) times it
+            const int n0 = -mt.y, n1 = -(mt.y << 2), n2 = -(mt.y << 4), n3 = -(mt.y * 85);
+            float* ppart = partial + (size_t)wi * 2 * S + sl + (lane >> 4) * S;
+            // a slot holds the unit as it lies in memory: atom (i, l) at 16 (i A + l), the scale quads after the atoms
+            const int ln = live ? lane : 0;
+            const int atom_stride = active * 16;
+            const int scale_off = active * 64 + (ln >> 1) * 8 - ln * 16;
+            for (int j = 0; j < n_rp; ++j) {
+                {   // wait (bounded) for the unit in slot cslot
+                    uint64_t* bar = bars + cslot;
+                    const int limit = failed ? kSpinLimitAfterFailure : kSpinLimit;
+                    int spins = 0;
+                    while (!mbar_try_wait(bar, phase)) {
+                        if (++spins >= limit) { failed = true; break; }
                     }
-                    ah[3] = dot_us(w[ww], xh[4 * i + ww], ah[3]);
-                    al[3] = dot_uu(w[ww], xl[4 * i + ww], al[3]);
                 }
-            }
-            const uint2 sc = *reinterpret_cast<const uint2*>(buf + scale_off);
-            const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));   // alpha1, alpha2 of row 0
-            const float2 s1 = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));   // ... of row 1
-            // Q0..Q2 = 4^f * sum_j t_j X_j of fields 0..2; the unmasked word minus those three is field 3's
-            const int Q0 = (ah[0] << 8) + al[0], Q1 = (ah[1] << 8) + al[1], Q2 = (ah[2] << 8) + al[2];
-            const int Q3 = (ah[3] << 8) + al[3] - Q0 - Q1 - Q2;
-            // lanes past the slice's columns redo lane 0 and are zeroed explicitly
-            float y0 = live ? c0 * fmaf(0.25f, s0.y * (float)Q1, s0.x * (float)Q0) : 0.f;
-            float y1 = live ? c1 * fmaf(0.25f, s1.y * (float)Q3, s1.x * (float)Q2) : 0.f;
-            // every lane has consumed the slot: lane 0 may refill it
-            __syncwarp();
-            issue();
-            if (++cslot == D) { cslot = 0; phase ^= 1u; }
-            // lanes 0-15 reduce row 0, lanes 16-31 row 1
-            const float send = (lane & 16) ? y0 : y1;
-            float v = ((lane & 16) ? y1 : y0) + __shfl_xor_sync(0xffffffffu, send, 16);
+                const unsigned char* buf = ring + cslot * kUnit2 + ln * 16;
+                // Fields 0..2 are masked out of each code word; the unmasked word gives the sum of all four fields
+                // (a byte is q0 + 4 q1 + 16 q2 + 64 q3 <= 170), so field 3 is "all" minus the other three.
+                int ah[4] = {0, 0, 0, 0};
+                int al[4] = {n0, n1, n2, n3};
 #pragma unroll
-            for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if ((lane & 15) == 0) *ppart = failed ? __int_as_float(0x7fc00000) : v;
-            ppart += (size_t)m * 2 * S;
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 cw = *reinterpret_cast<const uint4*>(buf + i * atom_stride);
+                    const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
+#pragma unroll
+                    for (int ww = 0; ww < 4; ++ww) {
+#pragma unroll
+                        for (int f = 0; f < 3; ++f) {
+                            const uint32_t mk = w[ww] & (0x03030303u << (2 * f));
+                            ah[f] = dot_us(mk, xh[4 * i + ww], ah[f]);
+                            al[f] = dot_uu(mk, xl[4 * i + ww], al[f]);
+                        }
+                        ah[3] = dot_us(w[ww], xh[4 * i + ww], ah[3]);
+                        al[3] = dot_uu(w[ww], xl[4 * i + ww], al[3]);
+                    }
+                }
+                const uint2 sc = *reinterpret_cast<const uint2*>(buf + scale_off);
+                const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));   // alpha1, alpha2 of row 0
+                const float2 s1 = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));   // ... of row 1
+                // Q0..Q2 = 4^f * sum_j t_j X_j of fields 0..2; the unmasked word minus those three is field 3's
+                const int Q0 = (ah[0] << 8) + al[0], Q1 = (ah[1] << 8) + al[1], Q2 = (ah[2] << 8) + al[2];
+                const int Q3 = (ah[3] << 8) + al[3] - Q0 - Q1 - Q2;
+                // lanes past the slice's columns redo lane 0 and are zeroed explicitly
+                float y0 = live ? c0 * fmaf(0.25f, s0.y * (float)Q1, s0.x * (float)Q0) : 0.f;
+                float y1 = live ? c1 * fmaf(0.25f, s1.y * (float)Q3, s1.x * (float)Q2) : 0.f;
+                // every lane has consumed the slot: lane 0 may refill it
+                __syncwarp();
+                issue();
+                if (++cslot == D) { cslot = 0; phase ^= 1u; }
+                // lanes 0-15 reduce row 0, lanes 16-31 row 1
+                const float send = (lane & 16) ? y0 : y1;
+                float v = ((lane & 16) ? y1 : y0) + __shfl_xor_sync(0xffffffffu, send, 16);
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if ((lane & 15) == 0) *ppart = failed ? __int_as_float(0x7fc00000) : v;
+                ppart += (size_t)m * 2 * S;
+            }
         }
+        if (!spec) break;
+        // Earlier work of the stream is complete after this wait: if x still reads as it did, the pass stands.
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        waited = true;
+        int stale = 0;
+#pragma unroll 4
+        for (int c = (int)threadIdx.x; c < nchunks; c += cthreads) {
+            const uint4 now = __ldcg(reinterpret_cast<const uint4*>(x) + c);
+            const uint4 was = first_read[c];
+            stale |= (now.x != was.x) | (now.y != was.y) | (now.z != was.z) | (now.w != was.w);
+        }
+        if (!__syncthreads_or(stale)) break;
     }
     if (failed && lane == 0) atomicExch(&g_gemv2_status, (int)PTQTP_ERR_CUDA);
     __syncthreads();
@@ -351,13 +364,13 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     }
 }
 
-size_t smem_bytes(const Layout2& L, int rows_cap, int warps, int depth) {
-    return smem_layout2(L.k, L.slices, rows_cap, warps, depth).total;
+size_t smem_bytes(const Layout2& L, int rows_cap, int warps, int depth, int speculate) {
+    return smem_layout2(L.k, L.slices, rows_cap, warps, depth, speculate).total;
 }
 
 template <int D>
 ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int grid, int warps,
-                      int rows_cap, size_t smem, cudaStream_t st) {
+                      int rows_cap, size_t smem, int speculate, cudaStream_t st) {
     auto kern = gemv2_kernel<D>;
     static thread_local size_t configured[64] = {};       // per device: largest dynamic smem already allowed
     int dev = 0;
@@ -379,12 +392,27 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
     cfg.numAttrs = overlap_enabled() ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, L, static_cast<const unsigned char*>(packed),
                                        reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap,
-                                       L.nrp / grid, L.nrp % grid, speculation_enabled() ? 1 : 0);
+                                       L.nrp / grid, L.nrp % grid, speculate);
     if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
     return PTQTP_OK;
 }
 
 }  // namespace
+
+// Address of the status word on the current device, for the other kernels that report through it.
+ptqtp_status gemv_status_word(int** out) {
+    static thread_local int* cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PTQTP_ERR_CUDA;
+    if (!cache[dev]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_gemv2_status);
+        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+        cache[dev] = static_cast<int*>(p);
+    }
+    *out = cache[dev];
+    return PTQTP_OK;
+}
 
 ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st) {
     cudaError_t e = cudaMemcpyFromSymbolAsync(status_host, g_gemv2_status, sizeof(int), 0, cudaMemcpyDeviceToHost, st);
@@ -392,34 +420,40 @@ ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st) {
     return PTQTP_OK;
 }
 
-ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps, int depth,
-                          cudaStream_t st) {
+// ctas_per_sm: CTAs of this launch per SM (0 = one).  The defaults keep a CTA small (4 to 8 warps, two ring slots
+// per warp) so that the CTAs of several consecutive launches are resident on an SM at once: under programmatic
+// dependent launch with speculative execution the head of one launch (fetching x) and the tail of another
+// (verifying x, reducing) then overlap the streaming of a third.  Measured on the LLaMA-3-8B shapes, 4 warps
+// beat 8 and 16 (6.9 / 7.3 / 8.5 us on 14336 x 4096).
+ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
+                          int ctas_per_sm, int depth, cudaStream_t st) {
     const int S = L.slices;
-    const int grid = min(sm_count(), L.nrp);
+    const int speculate = speculation_enabled() ? 1 : 0;
+    if (ctas_per_sm < 0 || ctas_per_sm > 4) return PTQTP_ERR_CONFIG;
+    if (warps < 0 || warps > kMaxWarps2) return PTQTP_ERR_CONFIG;
+    const int per_sm = ctas_per_sm ? ctas_per_sm : 1;
+    const int max_warps = kMaxWarps2 / per_sm;
+    const size_t budget = (size_t)(228 / per_sm - 1) * 1024;          // 228 KB per SM, 1 KB of it reserved per CTA
+    const int grid = min(per_sm * sm_count(), L.nrp);
     if (warps == 0) {
-        // A multiple of the slice count (every slice lane gets as many warps): about 16 warps when a CTA has
-        // many slice units to stream, about 8 when it has few (measured on the LLaMA-3 shapes).
+        // a multiple of the slice count (every slice lane gets as many warps): at least 4, at least 8 when a CTA
+        // streams many units, and all 16 when that is what it takes to give every slice a warp
         const long units_per_cta = (long)((L.nrp + grid - 1) / grid) * S;
-        const int target = units_per_cta >= 64 ? 16 : 8;
-        warps = S >= kMaxWarps2 ? kMaxWarps2 : S * max(1, (target + S / 2) / S);
-        if (warps > kMaxWarps2) warps = S * (kMaxWarps2 / S);
+        const int target = units_per_cta >= 256 ? 8 : 4;
+        warps = S >= max_warps ? max_warps : S * ((target + S - 1) / S);
+        if (warps > max_warps) warps = S * (max_warps / S);
     }
-    if (warps < 1 || warps > kMaxWarps2) return PTQTP_ERR_CONFIG;
+    if (warps < 1 || warps > max_warps) return PTQTP_ERR_CONFIG;
     const int rows_cap = 2 * ((L.nrp + grid - 1) / grid);
-    const size_t budget = 227 * 1024;
-    if (depth == 0) {
-        // measured: two slots per warp are best when a CTA streams many units, three when it has few
-        depth = (long)((L.nrp + grid - 1) / grid) * S >= 64 ? 2 : 3;
-        while (depth > 2 && smem_bytes(L, rows_cap, warps, depth) > budget) --depth;
-    }
-    const size_t smem = smem_bytes(L, rows_cap, warps, depth);
-    if (smem > budget) return depth > 2 || warps > 1 ? PTQTP_ERR_CONFIG : PTQTP_ERR_SHAPE;
+    if (depth == 0) depth = 2;
+    const size_t smem = smem_bytes(L, rows_cap, warps, depth, speculate);
+    if (smem > budget) return depth > 2 || warps > 1 || ctas_per_sm == 2 ? PTQTP_ERR_CONFIG : PTQTP_ERR_SHAPE;
     switch (depth) {
-        case 2: return launch_d<2>(L, packed, x, y, grid, warps, rows_cap, smem, st);
-        case 3: return launch_d<3>(L, packed, x, y, grid, warps, rows_cap, smem, st);
-        case 4: return launch_d<4>(L, packed, x, y, grid, warps, rows_cap, smem, st);
-        case 6: return launch_d<6>(L, packed, x, y, grid, warps, rows_cap, smem, st);
-        case 8: return launch_d<8>(L, packed, x, y, grid, warps, rows_cap, smem, st);
+        case 2: return launch_d<2>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
+        case 3: return launch_d<3>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
+        case 4: return launch_d<4>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
+        case 6: return launch_d<6>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
+        case 8: return launch_d<8>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
     }
     return PTQTP_ERR_CONFIG;
 }

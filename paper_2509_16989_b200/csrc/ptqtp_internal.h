@@ -98,7 +98,7 @@ ptqtp_status launch_pack2(const Layout2& L, const int8_t* T1, const int8_t* T2, 
 ptqtp_status launch_unpack2(const Layout2& L, const void* packed, int8_t* T1, int8_t* T2, uint16_t* a1,
                             uint16_t* a2, int32_t* dev_status, cudaStream_t st);
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
-                          int depth, cudaStream_t st);
+                          int ctas_per_sm, int depth, cudaStream_t st);
 ptqtp_status launch_skinny2(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y,
                             cudaStream_t st);
 size_t skinny3_workspace_bytes(int k, int m);
@@ -106,6 +106,10 @@ ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const u
                             cudaStream_t st);
 ptqtp_status static_workspace_address(void** out);
 ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st);
+ptqtp_status gemv_status_word(int** out);      // device address of the word copy_gemv2_status reads
+// 1 <= m <= 4 on the tensor-core path; PTQTP_ERR_SHAPE when (K, m) leaves no room for its ring in shared memory
+ptqtp_status launch_gemv3(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, int warps,
+                          int ctas_per_sm, int depth, cudaStream_t st);
 int sm_count();
 bool speculation_enabled();       // speculative read of x before the dependency wait (ptqtp_set_overlap(2))
 bool overlap_enabled();           // programmatic dependent launch of the GEMV kernels (ptqtp_set_overlap)

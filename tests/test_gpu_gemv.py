@@ -15,6 +15,10 @@ from gpu_util import FORMATS, assert_parity, dev, oracle_y, pack_case
 pytestmark = pytest.mark.gpu
 
 
+def dev_packed(c):
+    return pack_case(c, binding.FORMAT_V2)
+
+
 def run_gemv(c, fmt=None, **cfg):
     packed = pack_case(c, fmt)
     if cfg:
@@ -41,11 +45,13 @@ def test_format2_launch_configurations(warps, depth):
         c = make_case(N, K, seed=warps * 10 + depth)
         ref = oracle_y(c)
         packed = pack_case(c, binding.FORMAT_V2)
-        # shared memory: x as two byte planes + block records, the slice partials, one mbarrier and one
-        # 2176-byte slot per ring entry
+        # shared memory: x as two byte planes + block records, the first read of x (speculative execution is on
+        # by default), the slice partials, one mbarrier and one 2176-byte slot per ring entry
         S = -(-K // 2048)
-        rows_cap = 2 * -(-((N + 1) // 2) // min(148, (N + 1) // 2))
-        bar_off = -(-((K // 64) * 136 + rows_cap * S * 4) // 8) * 8
+        nrp = (N + 1) // 2
+        rows_cap = 2 * -(-nrp // min(148, nrp))
+        raw_off = -(-((K // 64) * 136) // 16) * 16
+        bar_off = -(-(raw_off + 2 * K + rows_cap * S * 4) // 8) * 8
         smem = -(-(bar_off + warps * depth * 8) // 16) * 16 + warps * depth * 2176
         if smem > 227 * 1024:
             with pytest.raises(binding.PtqtpError) as e:
@@ -57,10 +63,79 @@ def test_format2_launch_configurations(warps, depth):
         assert_parity(y.cpu().numpy(), ref, c["x"], "warps=%d depth=%d N=%d K=%d" % (warps, depth, N, K))
 
 
+@pytest.mark.parametrize("per_sm", [0, 1, 2])
+@pytest.mark.parametrize("warps,depth", [(0, 0), (4, 2), (8, 3), (7, 2), (2, 4)])
+def test_format2_ctas_per_sm(warps, depth, per_sm):
+    for N, K in ((300, 4096), (1000, 14336), (5, 2048), (2400, 1024), (4097, 6144)):
+        c = make_case(N, K, seed=warps + depth)
+        y = binding.ptqtp_gemv_cfg(pack_case(c, binding.FORMAT_V2), N, K, dev(c["x"]), k_split=warps, depth=depth,
+                                   ctas_per_sm=per_sm, fmt=binding.FORMAT_V2)
+        torch.cuda.synchronize()
+        assert_parity(y.cpu().numpy(), oracle_y(c), c["x"], "warps=%d depth=%d per_sm=%d N=%d K=%d" % (warps, depth, per_sm, N, K))
+
+
+@pytest.mark.parametrize("arith", [3, 4])
+@pytest.mark.parametrize("N,K", [(1, 128), (2, 256), (7, 1024), (8, 1152), (9, 2048), (31, 2176), (33, 3200), (130, 4096),
+                                 (257, 5120), (64, 14336), (1000, 6144), (37, 36864), (1190, 4096), (4736, 1024),
+                                 (2377, 8192)])
+def test_format2_both_kernels(N, K, arith):
+    # arith 3: masks + integer dot products on the CUDA cores; arith 4: int8 tensor-core MMAs
+    c = make_case(N, K, seed=100 + N)
+    assert_parity(run_gemv(c, binding.FORMAT_V2, arith=arith), oracle_y(c), c["x"], "arith=%d N=%d K=%d" % (arith, N, K))
+
+
+def _tensor_core_smem(N, K, warps, per_sm, depth):
+    # two byte planes of x (K + 64 each), group records, the quarter-slice partials, two mbarriers and four
+    # 2192-byte unit slots per stage for each team of four warps (the first read of x, which speculative execution
+    # keeps as well, is dropped when it does not fit)
+    teams = warps // 4
+    S, quads = -(-K // 2048), -(-((N + 1) // 2) // 4)
+    rows_cap = 8 * -(-quads // min(per_sm * 148, quads))
+    raw_off = -(-(2 * (K + 64) + (K // 128) * 8) // 16) * 16
+    bar_off = -(-(raw_off + rows_cap * 4 * S * 4) // 8) * 8
+    return -(-(bar_off + teams * depth * 16) // 16) * 16 + teams * depth * 4 * 2192
+
+
+@pytest.mark.parametrize("per_sm", [1, 2])
+@pytest.mark.parametrize("warps", [4, 8, 16])
+@pytest.mark.parametrize("depth", [2, 3, 4, 8])
+def test_format2_tensor_core_configurations(depth, warps, per_sm):
+    for N, K in ((67, 8192), (1000, 14336), (4, 2048), (2400, 4096), (5000, 1024)):
+        c = make_case(N, K, seed=depth)
+        fits = warps * per_sm <= 16 and _tensor_core_smem(N, K, warps, per_sm, depth) <= (228 // per_sm - 1) * 1024
+        if not fits:
+            with pytest.raises(binding.PtqtpError) as e:
+                binding.ptqtp_gemv_cfg(dev_packed(c), N, K, dev(c["x"]), k_split=warps, ctas_per_sm=per_sm, depth=depth,
+                                       arith=4, fmt=binding.FORMAT_V2)
+            assert e.value.status == binding.ERR_CONFIG
+            continue
+        y = binding.ptqtp_gemv_cfg(dev_packed(c), N, K, dev(c["x"]), k_split=warps, ctas_per_sm=per_sm, depth=depth,
+                                   arith=4, fmt=binding.FORMAT_V2)
+        torch.cuda.synchronize()
+        assert_parity(y.cpu().numpy(), oracle_y(c), c["x"],
+                      "depth=%d warps=%d per_sm=%d N=%d K=%d" % (depth, warps, per_sm, N, K))
+
+
+def test_format2_tensor_core_kernel_is_exact_on_integers():
+    # small integers, unit scales: every step of the integer path is exact, so the fp16 result must be too
+    N, K = 300, 4096
+    c = make_case(N, K, seed=9)
+    rng = np.random.default_rng(9)
+    c["x"] = rng.integers(-8, 9, K).astype(np.float16)
+    c["alpha1"] = np.full_like(c["alpha1"], 1.0)
+    c["alpha2"] = np.full_like(c["alpha2"], 0.5)
+    ref = oracle_y(c)
+    for arith in (3, 4):
+        y = run_gemv(c, binding.FORMAT_V2, arith=arith)
+        assert np.array_equal(y.astype(np.float64), ref.astype(np.float16).astype(np.float64)), arith
+
+
 def test_format2_rejects_format1_only_options():
     c = make_case(8, 1024, seed=1)
     packed = pack_case(c, binding.FORMAT_V2)
-    for bad in (dict(rows_per_warp=2), dict(ctas_per_sm=3), dict(arith=1), dict(k_split=17), dict(depth=5)):
+    for bad in (dict(rows_per_warp=2), dict(arith=1), dict(k_split=17), dict(depth=5),
+                dict(arith=4, k_split=7), dict(arith=4, depth=9), dict(arith=4, depth=1), dict(arith=4, ctas_per_sm=3),
+                dict(ctas_per_sm=5)):
         with pytest.raises(binding.PtqtpError) as e:
             binding.ptqtp_gemv_cfg(packed, 8, 1024, dev(c["x"]), fmt=binding.FORMAT_V2, **bad)
         assert e.value.status == binding.ERR_CONFIG
