@@ -36,7 +36,7 @@ UNIQUE_OF = {"q": "qo", "o": "qo", "k": "kv", "v": "kv", "gate": "gate_up", "up"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes in the ncu capture of the 14336x4096 launch of
 # the current GEMV kernel (profiles/gemv2_gate_up_14336x4096.md); set to None when the kernel changes
-DRAM_TRAFFIC_RATIO = None
+DRAM_TRAFFIC_RATIO = 31227904.0 / 31232000.0
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -433,6 +433,29 @@ def run_gpu(args):
                          "us_isolated_median": float(np.median(iso)), "buffers": nbuf}
             del bufs
         del flush
+        # the same step without any overlap of consecutive launches (plain launches, no speculative execution)
+        if graphs is not None:
+            old_level = binding.ptqtp_set_overlap(0)
+            try:
+                with torch.cuda.stream(stream):
+                    step(0)
+                    stream.synchronize()
+                    plain = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(plain, stream=stream):
+                        for r in range(R):
+                            step(r)
+                    plain.replay()
+                    stream.synchronize()
+                    e0.record(stream)
+                    for _ in range(20):
+                        plain.replay()
+                    e1.record(stream)
+                    stream.synchronize()
+                detail["step_without_overlap"] = {"us_per_layer": 1e3 * e0.elapsed_time(e1) / (20 * R),
+                                                  "what": "ptqtp_set_overlap(0): every launch waits for the one before it"}
+                del plain
+            finally:
+                binding.ptqtp_set_overlap(old_level)
 
     sampler.stop()
 
@@ -450,7 +473,9 @@ def run_gpu(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: steps rotate over %d layer copies (%d MB)"
                    % (R, R * STEP_WEIGHT_BYTES >> 20), "launch": "cuda graph" if graphs else "plain launches",
-                   "parallelism": "replicas only" if world > 1 else "1 gpu", "bytes_per_step": STEP_BYTES},
+                   "parallelism": "replicas only" if world > 1 else "1 gpu", "bytes_per_step": STEP_BYTES,
+                   "overlap": "library default (ptqtp_set_overlap level 2): programmatic dependent launch with "
+                              "speculative execution; the CTAs of consecutive launches share SMs"},
         "us_per_layer": 1e3 * ms_per_step,
         "weight_gbs": STEP_WEIGHT_BYTES / (ms_per_step * 1e-3) / 1e9,
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,

@@ -194,7 +194,8 @@ ptqtp_status ptqtp_gemv_host(const ptqtp_shape* shape, const void* packed, size_
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)shape->k_in * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
-    s = gemv_any(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
+    // between its two copies the kernel never overlaps another GEMV: it gets whole SMs
+    s = L.v2 ? launch_gemv2(L.l2, packed, x_dev, y_dev, -1, 0, 0, st) : gemv_any(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
     if (s != PTQTP_OK) return s;
     e = cudaMemcpyAsync(y_host, y_dev, (size_t)shape->n_out * 2, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }

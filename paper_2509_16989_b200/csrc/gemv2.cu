@@ -375,6 +375,13 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
     static thread_local size_t configured[64] = {};       // per device: largest dynamic smem already allowed
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    if (configured[dev] == 0) {
+        // every launch asks for the largest shared-memory carveout: consecutive launches with different
+        // carveouts cannot share an SM (it drains to be reconfigured), and these kernels make no use of L1
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+        configured[dev] = 1;
+    }
     if (smem > 48 * 1024 && smem > configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
@@ -420,6 +427,7 @@ ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st) {
     return PTQTP_OK;
 }
 
+// warps: per CTA, 0 = the default below, -1 = as many as fit (for a call that is known to run alone).
 // ctas_per_sm: CTAs of this launch per SM (0 = one).  The defaults keep a CTA small (4 to 8 warps, two ring slots
 // per warp) so that the CTAs of several consecutive launches are resident on an SM at once: under programmatic
 // dependent launch with speculative execution the head of one launch (fetching x) and the tail of another
@@ -430,12 +438,16 @@ ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* 
     const int S = L.slices;
     const int speculate = speculation_enabled() ? 1 : 0;
     if (ctas_per_sm < 0 || ctas_per_sm > 4) return PTQTP_ERR_CONFIG;
-    if (warps < 0 || warps > kMaxWarps2) return PTQTP_ERR_CONFIG;
+    if (warps < -1 || warps > kMaxWarps2) return PTQTP_ERR_CONFIG;
     const int per_sm = ctas_per_sm ? ctas_per_sm : 1;
     const int max_warps = kMaxWarps2 / per_sm;
     const size_t budget = (size_t)(228 / per_sm - 1) * 1024;          // 228 KB per SM, 1 KB of it reserved per CTA
     const int grid = min(per_sm * sm_count(), L.nrp);
-    if (warps == 0) {
+    if (warps == 0 && !overlap_enabled()) warps = -1;   // plain launches never share an SM
+    if (warps == -1) {
+        // the caller knows that the call runs alone (copies on both sides of it): one CTA takes the whole SM
+        warps = S >= max_warps ? max_warps : S * (max_warps / S);
+    } else if (warps == 0) {
         // a multiple of the slice count (every slice lane gets as many warps): at least 4, at least 8 when a CTA
         // streams many units, and all 16 when that is what it takes to give every slice a warp
         const long units_per_cta = (long)((L.nrp + grid - 1) / grid) * S;

@@ -449,6 +449,13 @@ ptqtp_status launch_gemv3(const Layout2& L, const void* packed, int m, const uin
     static thread_local size_t configured[64] = {};       // per device: largest dynamic smem already allowed
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    if (configured[dev] == 0) {
+        // every launch asks for the largest shared-memory carveout: consecutive launches with different
+        // carveouts cannot share an SM (it drains to be reconfigured), and these kernels make no use of L1
+        cudaError_t e = cudaFuncSetAttribute(gemv3_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+        configured[dev] = 1;
+    }
     if (smem > 48 * 1024 && smem > configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(gemv3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
