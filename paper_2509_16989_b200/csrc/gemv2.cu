@@ -81,22 +81,19 @@ __device__ __forceinline__ int dot_uu(uint32_t a, uint32_t x, int c) {
     return d;
 }
 
-// Convert 8 activations (one uint4 of fp16) to block fixed point and store them in shared memory.
-//   xhi, xlo : [K/64 blocks][16 words]  bytes of hi_j / lo_j in column order
+// Convert 16 activations (two uint4 of fp16: columns base .. base + 15) to block fixed point and store them.
+//   xhi, xlo : [K/64 blocks][16 words]  bytes of hi_j / lo_j in column order, 16-byte chunks permuted (see below)
 //   meta     : [K/64 blocks] (2^-s as float bits, sum_j X_j)
-// Eight adjacent threads share a 64-column block (8 columns each); the whole warp must call this.
-__device__ __noinline__ void convert_x8(uint4 raw, int base, bool valid, uint32_t* xhi, uint32_t* xlo, int2* meta) {
-    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+// Four adjacent threads share a 64-column block (16 columns each); the whole warp must call this.
+__device__ __noinline__ void convert_x16(uint4 ra, uint4 rb, int base, bool valid, uint32_t* xhi, uint32_t* xlo, int2* meta) {
+    const uint32_t rw[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
     // block maximum of |x| on the fp16 bit patterns (ordered like the values once the sign is cleared)
-    const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-    uint32_t mxb = 0u;
+    uint32_t m2 = 0u;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const uint32_t a = rw[e] & 0x7fff7fffu;
-        mxb = max(mxb, max(a & 0xffffu, a >> 16));
-    }
-#pragma unroll
-    for (int o = 1; o < 8; o <<= 1) mxb = max(mxb, __shfl_xor_sync(0xffffffffu, mxb, o));
+    for (int e = 0; e < 8; ++e) m2 = __vmaxu2(m2, rw[e] & 0x7fff7fffu);
+    uint32_t mxb = max(m2 & 0xffffu, m2 >> 16);
+    mxb = max(mxb, __shfl_xor_sync(0xffffffffu, mxb, 1));
+    mxb = max(mxb, __shfl_xor_sync(0xffffffffu, mxb, 2));
     // exponent of the block maximum, in [-24, 15] for finite inputs; subnormal fp16 (exponent field 0) are
     // integers times 2^-24
     int s = 0;
@@ -106,36 +103,37 @@ __device__ __noinline__ void convert_x8(uint4 raw, int base, bool valid, uint32_
         s = 14 - ex;
     }
     const float scale = __uint_as_float((uint32_t)(127 + s) << 23);
-    int X[8];
-    int sum = 0;
+    // x * 2^s is exact and below 2^15 in magnitude; adding 1.5 * 2^23 rounds it to the nearest integer (ties to
+    // even) and leaves that integer, as a 16-bit two's complement number, in the low 16 bits of the float
+    uint32_t B[16];
+    uint32_t sum = 0u;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const float2 v = __half22float2(h2[e]);
-        // x * 2^s is exact and below 2^15 in magnitude; adding 1.5 * 2^23 rounds it to the nearest integer
-        // (ties to even) and leaves that integer in the low mantissa bits
-        X[2 * e] = __float_as_int(fmaf(v.x, scale, 12582912.f)) - 0x4B400000;
-        X[2 * e + 1] = __float_as_int(fmaf(v.y, scale, 12582912.f)) - 0x4B400000;
-        sum += X[2 * e] + X[2 * e + 1];
+    for (int e = 0; e < 8; ++e) {
+        const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&rw[e]));
+        B[2 * e] = __float_as_uint(fmaf(v.x, scale, 12582912.f));
+        B[2 * e + 1] = __float_as_uint(fmaf(v.y, scale, 12582912.f));
+        sum += B[2 * e] + B[2 * e + 1];
     }
+    int isum = (int)(sum - 16u * 0x4B400000u);          // sum of the integers themselves
+    isum += __shfl_xor_sync(0xffffffffu, isum, 1);
+    isum += __shfl_xor_sync(0xffffffffu, isum, 2);
+    uint32_t hw[4], lw[4];
 #pragma unroll
-    for (int o = 1; o < 8; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    uint32_t hw[2], lw[2];
-#pragma unroll
-    for (int w = 0; w < 2; ++w) {
+    for (int w = 0; w < 4; ++w) {
         // byte 0 (lo) and byte 1 (hi) of four consecutive X gathered into one word each
-        const uint32_t lo01 = __byte_perm(X[4 * w], X[4 * w + 1], 0x0040), lo23 = __byte_perm(X[4 * w + 2], X[4 * w + 3], 0x0040);
-        const uint32_t hi01 = __byte_perm(X[4 * w], X[4 * w + 1], 0x0051), hi23 = __byte_perm(X[4 * w + 2], X[4 * w + 3], 0x0051);
+        const uint32_t lo01 = __byte_perm(B[4 * w], B[4 * w + 1], 0x0040), lo23 = __byte_perm(B[4 * w + 2], B[4 * w + 3], 0x0040);
+        const uint32_t hi01 = __byte_perm(B[4 * w], B[4 * w + 1], 0x0051), hi23 = __byte_perm(B[4 * w + 2], B[4 * w + 3], 0x0051);
         lw[w] = __byte_perm(lo01, lo23, 0x5410);
         hw[w] = __byte_perm(hi01, hi23, 0x5410);
     }
     if (valid) {
         // the four 16-byte chunks of a block are stored permuted (chunk v at v ^ swz) so that the lanes of a warp,
         // which each read a whole block with 128-bit loads, do not collide on shared-memory banks
-        const int blk = base >> 6, tt = (base >> 3) & 7;
-        const int pos = blk * 16 + (((tt >> 1) ^ ((blk >> 1) & 3)) << 2) + ((tt & 1) << 1);
-        *reinterpret_cast<uint2*>(xhi + pos) = make_uint2(hw[0], hw[1]);
-        *reinterpret_cast<uint2*>(xlo + pos) = make_uint2(lw[0], lw[1]);
-        if (tt == 0) meta[blk] = make_int2((int)((uint32_t)(127 - s) << 23), sum);
+        const int blk = base >> 6, v = (base >> 4) & 3;
+        const int pos = blk * 16 + ((v ^ ((blk >> 1) & 3)) << 2);
+        *reinterpret_cast<uint4*>(xhi + pos) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        *reinterpret_cast<uint4*>(xlo + pos) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+        if (v == 0) meta[blk] = make_int2((int)((uint32_t)(127 - s) << 23), isum);
     }
 }
 
@@ -188,7 +186,7 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     const int n_rp = idle ? 0 : max(0, (rp1 - rp0 - wi + m - 1) / m);
     const unsigned char* codes = packed + L.codes_off + (size_t)(rp0 + wi) * L.strip;
     const size_t rp_stride = (size_t)m * L.strip;
-    const int nchunks = L.k >> 3, cthreads = blockDim.x;
+    const int nchunks = L.k >> 3, nchunks16 = L.k >> 4, cthreads = blockDim.x;
 
     if (lane == 0) {
 #pragma unroll
@@ -230,18 +228,21 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
         pt = n_rp > 0 ? 0 : n_sl;
         pj = 0;
         psrc = codes + (size_t)sl_lane * kUnit2;
-        // x -> block fixed point in shared memory, four 8-column chunks per thread in flight.  Reads go to L2
+        // x -> block fixed point in shared memory, two 16-column chunks per thread in flight.  Reads go to L2
         // (ld.global.cg), the point of coherence, never through L1.  The first reads are issued before the ring
         // is filled (behind the fill they would wait for all of it); the packed planes do not depend on earlier
         // work of the stream, so the fill never waits for that work.
         bool filled = false;
-        for (int cb = (int)threadIdx.x; (cb & ~31) < nchunks; cb += 4 * cthreads) {
+        for (int cb = (int)threadIdx.x; (cb & ~31) < nchunks16; cb += 2 * cthreads) {
             uint4 r[4];
 #pragma unroll
-            for (int p = 0; p < 4; ++p) {
+            for (int p = 0; p < 2; ++p) {
                 const int c = cb + p * cthreads;
-                r[p] = make_uint4(0u, 0u, 0u, 0u);
-                if (c < nchunks) r[p] = __ldcg(reinterpret_cast<const uint4*>(x) + c);
+                r[2 * p] = r[2 * p + 1] = make_uint4(0u, 0u, 0u, 0u);
+                if (c < nchunks16) {
+                    r[2 * p] = __ldcg(reinterpret_cast<const uint4*>(x) + 2 * c);
+                    r[2 * p + 1] = __ldcg(reinterpret_cast<const uint4*>(x) + 2 * c + 1);
+                }
             }
             if (!filled) {
                 filled = true;
@@ -249,11 +250,11 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                 for (int d = 0; d < D; ++d) issue();
             }
 #pragma unroll
-            for (int p = 0; p < 4; ++p) {
+            for (int p = 0; p < 2; ++p) {
                 const int c = cb + p * cthreads;
-                if ((c & ~31) < nchunks) {
-                    if (spec && c < nchunks) first_read[c] = r[p];
-                    convert_x8(r[p], c << 3, c < nchunks, xhi, xlo, meta);
+                if ((c & ~31) < nchunks16) {
+                    if (spec && c < nchunks16) { first_read[2 * c] = r[2 * p]; first_read[2 * c + 1] = r[2 * p + 1]; }
+                    convert_x16(r[2 * p], r[2 * p + 1], c << 4, c < nchunks16, xhi, xlo, meta);
                 }
             }
         }
