@@ -122,20 +122,17 @@ __host__ __device__ inline Smem3 smem_layout3(int k, int m, int slices, int rows
     return s;
 }
 
-// Convert 8 activations (one uint4 of fp16, columns col..col+7 of batch row mi) to block fixed point and store
-// them.  Sixteen adjacent threads share a 128-column group; the whole warp must call this.
-__device__ __noinline__ void convert3_x8(uint4 raw, int mi, int col, bool valid, int k, unsigned char* xs, int2* meta) {
-    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+// Convert 16 activations (two uint4 of fp16, columns col..col+15 of batch row mi) to block fixed point and store
+// them.  Eight adjacent threads share a 128-column group; the whole warp must call this.
+__device__ __noinline__ void convert3_x16(uint4 ra, uint4 rb, int mi, int col, bool valid, int k, unsigned char* xs, int2* meta) {
+    const uint32_t rw[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
     // group maximum of |x| on the fp16 bit patterns (ordered like the values once the sign is cleared)
-    const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-    uint32_t mxb = 0u;
+    uint32_t m2 = 0u;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const uint32_t a = rw[e] & 0x7fff7fffu;
-        mxb = max(mxb, max(a & 0xffffu, a >> 16));
-    }
+    for (int e = 0; e < 8; ++e) m2 = __vmaxu2(m2, rw[e] & 0x7fff7fffu);
+    uint32_t mxb = max(m2 & 0xffffu, m2 >> 16);
 #pragma unroll
-    for (int o = 1; o < 16; o <<= 1) mxb = max(mxb, __shfl_xor_sync(0xffffffffu, mxb, o));
+    for (int o = 1; o < 8; o <<= 1) mxb = max(mxb, __shfl_xor_sync(0xffffffffu, mxb, o));
     // exponent of the maximum, in [-24, 15] for finite inputs; subnormal fp16 are integers times 2^-24
     int s = 0;
     if (mxb != 0u) {
@@ -144,39 +141,39 @@ __device__ __noinline__ void convert3_x8(uint4 raw, int mi, int col, bool valid,
         s = 13 - ex;                                   // group maximum in [2^13, 2^14): high byte within [-64, 64]
     }
     const float scale = __uint_as_float((uint32_t)(127 + s) << 23);
-    int H[8], Lo[8];
-    int sum = 0;
+    // x * 2^s is exact and below 2^14 in magnitude; adding 1.5 * 2^23 rounds it to the nearest integer (ties to
+    // even) and leaves that integer X, as a 16-bit two's complement number, in the low 16 bits of the float.
+    // X = 256 hi + lo with both bytes signed: lo is byte 0 of X, hi is byte 1 of X + 128.
+    uint32_t B[16];
+    uint32_t sum = 0u;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const float2 v = __half22float2(h2[e]);
-        // x * 2^s is exact and below 2^14 in magnitude; adding 1.5 * 2^23 rounds it to the nearest integer (ties
-        // to even) and leaves that integer in the low mantissa bits
-        const int X0 = __float_as_int(fmaf(v.x, scale, 12582912.f)) - 0x4B400000;
-        const int X1 = __float_as_int(fmaf(v.y, scale, 12582912.f)) - 0x4B400000;
-        sum += X0 + X1;
-        Lo[2 * e] = (int)(signed char)(X0 & 0xff);
-        Lo[2 * e + 1] = (int)(signed char)(X1 & 0xff);
-        H[2 * e] = (X0 - Lo[2 * e]) >> 8;
-        H[2 * e + 1] = (X1 - Lo[2 * e + 1]) >> 8;
+    for (int e = 0; e < 8; ++e) {
+        const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&rw[e]));
+        B[2 * e] = __float_as_uint(fmaf(v.x, scale, 12582912.f));
+        B[2 * e + 1] = __float_as_uint(fmaf(v.y, scale, 12582912.f));
+        sum += B[2 * e] + B[2 * e + 1];
     }
+    int isum = (int)(sum - 16u * 0x4B400000u);          // sum of the integers themselves
 #pragma unroll
-    for (int o = 1; o < 16; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    uint32_t hw[2], lw[2];
+    for (int o = 1; o < 8; o <<= 1) isum += __shfl_xor_sync(0xffffffffu, isum, o);
+    uint32_t hw[4], lw[4];
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
-        lw[q] = __byte_perm(__byte_perm(Lo[4 * q], Lo[4 * q + 1], 0x0040), __byte_perm(Lo[4 * q + 2], Lo[4 * q + 3], 0x0040), 0x5410);
-        hw[q] = __byte_perm(__byte_perm(H[4 * q], H[4 * q + 1], 0x0040), __byte_perm(H[4 * q + 2], H[4 * q + 3], 0x0040), 0x5410);
+    for (int w = 0; w < 4; ++w) {
+        const uint32_t h0 = B[4 * w] + 0x80u, h1 = B[4 * w + 1] + 0x80u, h2 = B[4 * w + 2] + 0x80u, h3 = B[4 * w + 3] + 0x80u;
+        lw[w] = __byte_perm(__byte_perm(B[4 * w], B[4 * w + 1], 0x0040), __byte_perm(B[4 * w + 2], B[4 * w + 3], 0x0040), 0x5410);
+        hw[w] = __byte_perm(__byte_perm(h0, h1, 0x0051), __byte_perm(h2, h3, 0x0051), 0x5410);
     }
     if (valid) {
-        // columns col..col+3 are word r = (col % 64) / 16 of lane t = (col % 16) / 4, columns col+4..col+7 of lane t + 1
+        // columns col + 4 t .. col + 4 t + 3 are word r = (col % 64) / 16 of lane t of their 64-column block
         const int c0 = col & 63;
-        unsigned char* hi = xs + (size_t)(2 * mi) * (k + kPlanePad) + (col - c0) + ((c0 & 15) >> 2) * 16 + (c0 >> 4) * 4;
+        unsigned char* hi = xs + (size_t)(2 * mi) * (k + kPlanePad) + (col - c0) + (c0 >> 4) * 4;
         unsigned char* lo = hi + k + kPlanePad;
-        *reinterpret_cast<uint32_t*>(hi) = hw[0];
-        *reinterpret_cast<uint32_t*>(hi + 16) = hw[1];
-        *reinterpret_cast<uint32_t*>(lo) = lw[0];
-        *reinterpret_cast<uint32_t*>(lo + 16) = lw[1];
-        if (((col >> 3) & 15) == 0) meta[mi * (k / kGroupCols) + (col >> 7)] = make_int2((int)((uint32_t)(127 - s) << 23), sum);
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            *reinterpret_cast<uint32_t*>(hi + 16 * w) = hw[w];
+            *reinterpret_cast<uint32_t*>(lo + 16 * w) = lw[w];
+        }
+        if (((col >> 4) & 7) == 0) meta[mi * (k / kGroupCols) + (col >> 7)] = make_int2((int)((uint32_t)(127 - s) << 23), isum);
     }
 }
 
@@ -209,7 +206,7 @@ gemv3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     const int nq = q_base + ((int)blockIdx.x < q_rem ? 1 : 0);
     const int T = nq * S;
     const int t0 = team * T / teams, ntask = (team + 1) * T / teams - t0;
-    const int chunks_per_row = L.k >> 3, nchunks = m * chunks_per_row;
+    const int nchunks = m * (L.k >> 3), chunks16_per_row = L.k >> 4, nchunks16 = m * chunks16_per_row;
     const unsigned char* codes = packed + L.codes_off;
 
     if ((int)threadIdx.x < teams * depth) {
@@ -271,25 +268,28 @@ gemv3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
         pq = t0 - ps * nq;
         produce();
         produce();
-        // x -> block fixed point in shared memory, four 8-column chunks per thread in flight.  Reads go to L2
+        // x -> block fixed point in shared memory, two 16-column chunks per thread in flight.  Reads go to L2
         // (ld.global.cg), the point of coherence, never through L1.
-        for (int cb = (int)threadIdx.x; (cb & ~31) < nchunks; cb += 4 * cthreads) {
+        for (int cb = (int)threadIdx.x; (cb & ~31) < nchunks16; cb += 2 * cthreads) {
             uint4 r[4];
 #pragma unroll
-            for (int p = 0; p < 4; ++p) {
+            for (int p = 0; p < 2; ++p) {
                 const int c = cb + p * cthreads;
-                r[p] = make_uint4(0u, 0u, 0u, 0u);
-                if (c < nchunks) r[p] = __ldcg(reinterpret_cast<const uint4*>(X) + c);
+                r[2 * p] = r[2 * p + 1] = make_uint4(0u, 0u, 0u, 0u);
+                if (c < nchunks16) {
+                    r[2 * p] = __ldcg(reinterpret_cast<const uint4*>(X) + 2 * c);
+                    r[2 * p + 1] = __ldcg(reinterpret_cast<const uint4*>(X) + 2 * c + 1);
+                }
             }
             if (cb == (int)threadIdx.x)
                 for (int d = 2; d < depth; ++d) produce();
 #pragma unroll
-            for (int p = 0; p < 4; ++p) {
+            for (int p = 0; p < 2; ++p) {
                 const int c = cb + p * cthreads;
-                if ((c & ~31) < nchunks) {
-                    if (spec && c < nchunks) first_read[c] = r[p];
-                    const int mi = c / chunks_per_row;
-                    convert3_x8(r[p], mi, (c - mi * chunks_per_row) << 3, c < nchunks, L.k, xs, meta);
+                if ((c & ~31) < nchunks16) {
+                    if (spec && c < nchunks16) { first_read[2 * c] = r[2 * p]; first_read[2 * c + 1] = r[2 * p + 1]; }
+                    const int mi = c / chunks16_per_row;
+                    convert3_x16(r[2 * p], r[2 * p + 1], mi, (c - mi * chunks16_per_row) << 4, c < nchunks16, L.k, xs, meta);
                 }
             }
         }
