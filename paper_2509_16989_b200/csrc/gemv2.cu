@@ -51,22 +51,23 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+// (the mbarriers and ring slots are addressed by their 32-bit shared-memory addresses)
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
 // Bulk copy global -> this CTA's shared memory, completion counted in bytes on an mbarrier (no multicast).
-__device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 // d = c + sum_b u8(a.b) * s8(x.b)   and   d = c + sum_b u8(a.b) * u8(x.b)
@@ -195,21 +196,23 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     }
     __syncwarp();
 
-    // producer (lane 0): slice pass pt, row pair pj, source of the next unit, ring slot
-    int pt = 0, pj = 0, pslot = 0;
+    // producer (lane 0): slice pass pt, row pairs left in it, source and size of the next unit, ring slot
+    const uint32_t bars_a = smem_u32(bars), ring_a = smem_u32(ring);
+    int pt = 0, pleft = 0, pslot = 0;
+    uint32_t pbytes = 0;
     const unsigned char* psrc = codes;
     auto issue = [&]() {
         if (pt < n_sl) {
             if (lane == 0) {
-                const uint32_t bytes = (sl_lane + pt * Wc) == S - 1 ? (uint32_t)L.last_unit : (uint32_t)kUnit2;
-                mbar_expect_tx(bars + pslot, bytes);
-                bulk_copy_g2s(ring + pslot * kUnit2, psrc, bytes, bars + pslot);
+                mbar_expect_tx(bars_a + 8 * pslot, pbytes);
+                bulk_copy_g2s(ring_a + pslot * kUnit2, psrc, pbytes, bars_a + 8 * pslot);
             }
             psrc += rp_stride;
-            if (++pj == n_rp) {
-                pj = 0;
+            if (--pleft == 0) {
                 ++pt;
+                pleft = n_rp;
                 psrc = codes + (size_t)(sl_lane + pt * Wc) * kUnit2;
+                pbytes = (sl_lane + pt * Wc) == S - 1 ? (uint32_t)L.last_unit : (uint32_t)kUnit2;
             }
         }
         pslot = pslot + 1 == D ? 0 : pslot + 1;
@@ -226,8 +229,9 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
             waited = true;
         }
         pt = n_rp > 0 ? 0 : n_sl;
-        pj = 0;
+        pleft = n_rp;
         psrc = codes + (size_t)sl_lane * kUnit2;
+        pbytes = sl_lane == S - 1 ? (uint32_t)L.last_unit : (uint32_t)kUnit2;
         // x -> block fixed point in shared memory, two 16-column chunks per thread in flight.  Reads go to L2
         // (ld.global.cg), the point of coherence, never through L1.  The first reads are issued before the ring
         // is filled (behind the fill they would wait for all of it); the packed planes do not depend on earlier
@@ -290,11 +294,11 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
             const int atom_stride = active * 16;
             const int scale_off = active * 64 + (ln >> 1) * 8 - ln * 16;
             for (int j = 0; j < n_rp; ++j) {
-                {   // wait (bounded) for the unit in slot cslot
-                    uint64_t* bar = bars + cslot;
+                // wait (bounded) for the unit in slot cslot; it has normally arrived long ago
+                if (!mbar_try_wait(bars_a + 8 * cslot, phase)) {
                     const int limit = failed ? kSpinLimitAfterFailure : kSpinLimit;
                     int spins = 0;
-                    while (!mbar_try_wait(bar, phase)) {
+                    while (!mbar_try_wait(bars_a + 8 * cslot, phase)) {
                         if (++spins >= limit) { failed = true; break; }
                     }
                 }
@@ -325,9 +329,10 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                 // Q0..Q2 = 4^f * sum_j t_j X_j of fields 0..2; the unmasked word minus those three is field 3's
                 const int Q0 = (ah[0] << 8) + al[0], Q1 = (ah[1] << 8) + al[1], Q2 = (ah[2] << 8) + al[2];
                 const int Q3 = (ah[3] << 8) + al[3] - Q0 - Q1 - Q2;
-                // lanes past the slice's columns redo lane 0 and are zeroed explicitly
-                float y0 = live ? c0 * fmaf(0.25f, s0.y * (float)Q1, s0.x * (float)Q0) : 0.f;
-                float y1 = live ? c1 * fmaf(0.25f, s1.y * (float)Q3, s1.x * (float)Q2) : 0.f;
+                // lanes past the slice's columns redo lane 0 and contribute zero
+                // (their block scale c0 is zero and the unit they read is real data, so their products are zero)
+                float y0 = c0 * fmaf(0.25f, s0.y * (float)Q1, s0.x * (float)Q0);
+                float y1 = c1 * fmaf(0.25f, s1.y * (float)Q3, s1.x * (float)Q2);
                 // every lane has consumed the slot: lane 0 may refill it
                 __syncwarp();
                 issue();
