@@ -167,7 +167,9 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     const Smem2 sm = smem_layout2(L.k, L.slices, rows_cap, warps, D, speculate);
     uint4* first_read = reinterpret_cast<uint4*>(smem + sm.raw_off);        // x as read before the dependency wait
     float* partial = reinterpret_cast<float*>(smem + sm.partial_off);       // [rows_cap][slices]
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // (the shuffle tells the compiler that the warp index is the same in all lanes: what derives from it can live
+    // in uniform registers, which the bulk-copy instruction wants)
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bar_off) + warp * D;
     unsigned char* ring = smem + sm.ring_off + (size_t)warp * D * kUnit2;
 
