@@ -45,10 +45,13 @@
  * Packed format 2 (same storage model; laid out for integer dot products: one mask yields four
  * byte-sized codes of four consecutive columns, see ptqtp_gemv):
  *   [0, 256)            header as above with format(2); the K_pad slot holds 2048 * ceil(K/2048) and the
- *                       scales_offset slot holds the row-pair stride in bytes.
+ *                       scales_offset slot holds the bytes of one row pair over all slices.
  *   body  (at 256)      ceil(N/2) row pairs, row pair p = rows 2p and 2p+1 (a missing row 2p+1 is stored
- *                       as trit 0 with scales 0).  A row pair is a strip of ceil(K/2048) slice units, slice s
- *                       covering columns 2048 s .. min(K, 2048 (s+1)) - 1 with A = columns/64 lane blocks:
+ *                       as trit 0 with scales 0), times ceil(K/2048) slices, slice s covering columns
+ *                       2048 s .. min(K, 2048 (s+1)) - 1.  Slice-major: the slice units of slice 0 for row pairs
+ *                       0, 1, 2, ... lie one after the other, then those of slice 1, and so on (a kernel that
+ *                       walks the rows of one slice reads one contiguous run).  A slice unit, with A =
+ *                       columns/64 lane blocks:
  *                         codes   4 * A atoms of 16 bytes; atom (i, l), i = 0..3, l = 0..A-1, at byte
  *                                 16 * (i * A + l), covers the 16 columns 2048 s + 64 l + 16 i + e, e = 0..15,
  *                                 one byte per column (byte e): bits [1:0] = code of (row 2p, plane 1),

@@ -14,10 +14,10 @@ one fp16 scale per plane per 128-column group):
                    (zero for padding groups).
 
 Format 2 (same header with format = 2; the K_pad slot holds 2048 * ceil(K/2048), the scales-offset slot the
-row-pair stride in bytes):
+bytes of one row pair over all slices):
 
-  body             for each row pair p (rows 2p, 2p+1; a missing odd row counts as trit 0, scales 0), for each
-                   slice s of up to 2048 columns with A = columns/64 lane blocks: 4*A atoms of 16 bytes, atom
+  body             for each slice s of up to 2048 columns, for each row pair p (rows 2p, 2p+1; a missing odd row
+                   counts as trit 0, scales 0), one unit with A = columns/64 lane blocks: 4*A atoms of 16 bytes, atom
                    (i, l) at byte 16*(i*A + l) holding columns 2048 s + 64 l + 16 i + e (e = 0..15), one byte
                    per column = code(2p, plane 1) | code(2p, plane 2) << 2 | code(2p+1, plane 1) << 4
                    | code(2p+1, plane 2) << 6; then A/2 quads of 4 little-endian u16 (alpha1[2p], alpha2[2p],
@@ -139,15 +139,17 @@ def layout_v2(N, K):
         raise ValueError("N > 0 and K a positive multiple of 128 required")
     nrp = (N + 1) // 2
     slices = (K + 2047) // 2048
-    units = []                                   # (first column, columns, byte offset in the strip, bytes)
+    units = []                                   # (first column, columns, byte offset of the slice's run, unit bytes)
     off = 0
+    strip = 0
     for sl in range(slices):
         cols = min(2048, K - 2048 * sl)
         size = -(-(cols + cols // 16) // 16) * 16
         units.append((2048 * sl, cols, off, size))
-        off += size
-    return dict(N=N, K=K, nrp=nrp, slices=slices, units=units, strip=off, codes_off=HEADER_BYTES,
-                total=HEADER_BYTES + nrp * off)
+        off += nrp * size                        # slice-major: the units of a slice for all row pairs are contiguous
+        strip += size
+    return dict(N=N, K=K, nrp=nrp, slices=slices, units=units, strip=strip, codes_off=HEADER_BYTES,
+                total=HEADER_BYTES + off)
 
 
 def pack_reference_v2(T1, T2, alpha1, alpha2):
@@ -171,13 +173,13 @@ def pack_reference_v2(T1, T2, alpha1, alpha2):
     hdr = MAGIC + struct.pack("<IIiiiiQQQ", 1, 2, N, K, 128, 2048 * L["slices"], L["codes_off"], L["strip"],
                               L["total"])
     blob[:len(hdr)] = np.frombuffer(hdr, dtype=np.uint8)
-    body = blob[L["codes_off"]:].reshape(nrp, L["strip"])
     for c0, cols, off, size in L["units"]:
         A = cols // 64
+        run = blob[L["codes_off"] + off:L["codes_off"] + off + nrp * size].reshape(nrp, size)   # one unit per row pair
         atoms = col_byte[:, c0:c0 + cols].reshape(nrp, A, 4, 16)   # [row pair, lane block, i, e]
-        body[:, off:off + 4 * A * 16] = atoms.transpose(0, 2, 1, 3).reshape(nrp, -1)
+        run[:, :4 * A * 16] = atoms.transpose(0, 2, 1, 3).reshape(nrp, -1)
         g0 = c0 // 128
-        body[:, off + 64 * A:off + 64 * A + 4 * A] = (
+        run[:, 64 * A:64 * A + 4 * A] = (
             np.ascontiguousarray(quads[:, g0:g0 + A // 2]).reshape(nrp, -1).view(np.uint8))
     return blob
 
@@ -197,17 +199,16 @@ def unpack_reference_v2(blob):
     if blob.size < L["total"]:
         raise ValueError("blob too small")
     nrp = L["nrp"]
-    body = blob[L["codes_off"]:L["total"]].reshape(nrp, L["strip"])
     col_byte = np.zeros((nrp, K), dtype=np.uint8)
     quads = np.zeros((nrp, K // 128, 4), dtype="<u2")
     for c0, cols, off, size in L["units"]:
         A = cols // 64
-        atoms = body[:, off:off + 4 * A * 16].reshape(nrp, 4, A, 16)
+        run = blob[L["codes_off"] + off:L["codes_off"] + off + nrp * size].reshape(nrp, size)   # one unit per row pair
+        atoms = run[:, :4 * A * 16].reshape(nrp, 4, A, 16)
         col_byte[:, c0:c0 + cols] = atoms.transpose(0, 2, 1, 3).reshape(nrp, cols)
         g0 = c0 // 128
-        quads[:, g0:g0 + A // 2] = np.ascontiguousarray(body[:, off + 64 * A:off + 68 * A]).view("<u2").reshape(
-            nrp, A // 2, 4)
-        if np.any(body[:, off + 68 * A:off + size] != 0):
+        quads[:, g0:g0 + A // 2] = np.ascontiguousarray(run[:, 64 * A:68 * A]).view("<u2").reshape(nrp, A // 2, 4)
+        if np.any(run[:, 68 * A:size] != 0):
             raise ValueError("unit padding must be zero")
     planes = []
     for plane in range(2):

@@ -57,17 +57,17 @@ static int default_gemv_arith() { return 3; }
 static ptqtp_status gemv_any(const AnyLayout& L, const void* packed, const uint16_t* x, uint16_t* y, int p0, int p1,
                              int p2, int p3, int p4, cudaStream_t st) {
     if (L.v2) {
-        if (p0 != 0 || (p4 != -1 && p4 != 3 && p4 != 4)) return PTQTP_ERR_CONFIG;
+        if ((p4 != -1 && p4 != 3 && p4 != 4) || (p0 != 0 && p4 == 4)) return PTQTP_ERR_CONFIG;
         if (p4 == 4) {                       // tensor-core kernel
             const ptqtp_status s = launch_gemv3(L.l2, packed, 1, x, y, p1, p2, p3, st);
             return s == PTQTP_ERR_SHAPE ? PTQTP_ERR_CONFIG : s;
         }
         if (p2 > 4) return PTQTP_ERR_CONFIG;
-        if (p4 == -1 && p1 == 0 && p2 == 0 && p3 == 0 && default_gemv_arith() == 4) {
+        if (p4 == -1 && p0 == 0 && p1 == 0 && p2 == 0 && p3 == 0 && default_gemv_arith() == 4) {
             const ptqtp_status s = launch_gemv3(L.l2, packed, 1, x, y, 0, 0, 0, st);
             if (s != PTQTP_ERR_SHAPE) return s;          // very long K: the CUDA-core kernel takes it
         }
-        return launch_gemv2(L.l2, packed, x, y, p1, p2, p3, st);
+        return launch_gemv2(L.l2, packed, x, y, p1, p2, p3, p0, st);
     }
     return launch_gemv(L.l1, packed, x, y, p0, p1, p2, p3, p4, st);
 }
@@ -143,7 +143,7 @@ ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, siz
             const ptqtp_status s4 = launch_gemv3(L.l2, packed, m, X, Y, 0, 0, 0, st);
             if (s4 != PTQTP_ERR_SHAPE) return s4;
         }
-        return m == 1 ? launch_gemv2(L.l2, packed, X, Y, 0, 0, 0, st) : launch_skinny2(L.l2, packed, m, X, Y, st);
+        return m == 1 ? launch_gemv2(L.l2, packed, X, Y, 0, 0, 0, 0, st) : launch_skinny2(L.l2, packed, m, X, Y, st);
     }
     return launch_gemm_skinny(L.l1, packed, m, X, Y, st);
 }
@@ -195,7 +195,7 @@ ptqtp_status ptqtp_gemv_host(const ptqtp_shape* shape, const void* packed, size_
     cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)shape->k_in * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
     // between its two copies the kernel never overlaps another GEMV: it gets whole SMs
-    s = L.v2 ? launch_gemv2(L.l2, packed, x_dev, y_dev, -1, 0, 0, st) : gemv_any(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
+    s = L.v2 ? launch_gemv2(L.l2, packed, x_dev, y_dev, -1, 0, 0, 0, st) : gemv_any(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
     if (s != PTQTP_OK) return s;
     e = cudaMemcpyAsync(y_host, y_dev, (size_t)shape->n_out * 2, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }

@@ -12,14 +12,15 @@
 //     byte).  fp16 values within 2^-5 of the block maximum are represented exactly; smaller ones are rounded
 //     to 2^-16 of the maximum.  All sums over a lane block are exact int32.
 //   * sum_j t_j X_j = sum_j q_j X_j - sum_j X_j (q = t + 1): the low accumulators start at minus the block sum.
-//   * A CTA owns a contiguous range of row pairs.  Warp w is bound to the 2048-column slice (w mod S) and keeps
-//     that slice's X (32 registers per lane) for its whole life; lanes own 64 consecutive columns, so a lane's
-//     four accumulator pairs (2 rows x 2 planes) see one scale group half and get the group's scales
-//     (the method's only multiplies) in an fp32 epilogue.
-//   * Each warp streams its slice units (2048 code bytes + 128 scale bytes, contiguous in HBM) through a
-//     private shared-memory ring: one bulk copy (cp.async.bulk, no multicast) per unit, issued by lane 0 and
-//     completed on an mbarrier, several units in flight, the first ones issued before x is fetched.  Bulk
-//     copies cost no load/store-unit time, which matters because the whole CTA waits for the fetch of x.
+//   * A CTA owns a contiguous range of row pairs.  Warp w is bound to the 2048-column slice (w mod S), takes a
+//     contiguous share of the CTA's row pairs and keeps the slice's X (32 registers per lane) while it stays
+//     there; lanes own 64 consecutive columns, so a lane's four accumulator pairs (2 rows x 2 planes) see one
+//     scale group half and get the group's scales (the method's only multiplies) in an fp32 epilogue.
+//   * The slice units of consecutive row pairs (2048 code bytes + 128 scale bytes each) are contiguous in HBM.
+//     Each warp streams its run of units through a private shared-memory ring: one bulk copy (cp.async.bulk,
+//     no multicast) per RU units, issued by lane 0 and completed on an mbarrier, several copies in flight.
+//     Issuing a copy and waiting for it cost about 40 instructions, which is why a copy brings several units.
+//     Bulk copies cost no load/store-unit time.
 //     Every wait on an mbarrier is bounded: if one gives up the warp writes NaN rows, records an error in a
 //     device status word (ptqtp_kernel_status) and still runs to the end.
 //   * Rows are reduced over the lanes by shuffles, over the slices through shared memory in a fixed order
@@ -140,21 +141,21 @@ __device__ __noinline__ void convert_x16(uint4 ra, uint4 rb, int base, bool vali
 
 // Shared memory: x as two byte planes and block records, the first read of x (fp16 as read, only when executing
 // speculatively), the per-slice partial sums, one mbarrier per ring slot, then the ring (one slice unit, kUnit2
-// bytes, per slot; D slots per warp).
+// bytes, RU of them per slot; D slots per warp).
 struct Smem2 {
     size_t raw_off, partial_off, bar_off, ring_off, total;
 };
-__host__ __device__ inline Smem2 smem_layout2(int k, int slices, int rows_cap, int warps, int depth, int speculate) {
+__host__ __device__ inline Smem2 smem_layout2(int k, int slices, int rows_cap, int warps, int depth, int ru, int speculate) {
     Smem2 m;
     m.raw_off = ((size_t)(k / kLane2) * 136 + 15) / 16 * 16;
     m.partial_off = m.raw_off + (speculate ? (size_t)2 * k : 0);
     m.bar_off = (m.partial_off + (size_t)rows_cap * slices * 4 + 7) / 8 * 8;
     m.ring_off = (m.bar_off + (size_t)warps * depth * 8 + 15) / 16 * 16;
-    m.total = m.ring_off + (size_t)warps * depth * kUnit2;
+    m.total = m.ring_off + (size_t)warps * depth * ru * kUnit2;
     return m;
 }
 
-template <int D>
+template <int D, int RU>
 __global__ void __launch_bounds__(kMaxThreads2, 1)
 gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
              __half* __restrict__ y, int rows_cap, int rp_base, int rp_rem, int speculate) {
@@ -164,14 +165,15 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     uint32_t* xlo = xhi + nblk * 16;
     int2* meta = reinterpret_cast<int2*>(xlo + nblk * 16);
     const int warps = blockDim.x >> 5;
-    const Smem2 sm = smem_layout2(L.k, L.slices, rows_cap, warps, D, speculate);
+    const Smem2 sm = smem_layout2(L.k, L.slices, rows_cap, warps, D, RU, speculate);
     uint4* first_read = reinterpret_cast<uint4*>(smem + sm.raw_off);        // x as read before the dependency wait
     float* partial = reinterpret_cast<float*>(smem + sm.partial_off);       // [rows_cap][slices]
     // (the shuffle tells the compiler that the warp index is the same in all lanes: what derives from it can live
     // in uniform registers, which the bulk-copy instruction wants)
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bar_off) + warp * D;
-    unsigned char* ring = smem + sm.ring_off + (size_t)warp * D * kUnit2;
+    constexpr int kSlot = RU * kUnit2;                 // a ring slot holds the RU units of one copy
+    unsigned char* ring = smem + sm.ring_off + (size_t)warp * D * kSlot;
 
     // Let the next kernel on the stream start while this one runs.
     asm volatile("griddepcontrol.launch_dependents;");
@@ -186,9 +188,11 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     const int sl_lane = warp % Wc, wi = warp / Wc;
     const bool idle = wi >= m;
     const int n_sl = idle ? 0 : (S - sl_lane + Wc - 1) / Wc;
-    const int n_rp = idle ? 0 : max(0, (rp1 - rp0 - wi + m - 1) / m);
-    const unsigned char* codes = packed + L.codes_off + (size_t)(rp0 + wi) * L.strip;
-    const size_t rp_stride = (size_t)m * L.strip;
+    // the m warps of a slice lane split the CTA's row pairs into contiguous runs (balanced +-1)
+    const int n_cta = rp1 - rp0;
+    const int rpw = rp0 + (idle ? 0 : wi * (n_cta / m) + min(wi, n_cta % m));
+    const int n_rp = idle ? 0 : n_cta / m + (wi < n_cta % m ? 1 : 0);
+    const unsigned char* codes = packed + L.codes_off;
     const int nchunks = L.k >> 3, nchunks16 = L.k >> 4, cthreads = blockDim.x;
 
     if (lane == 0) {
@@ -198,22 +202,25 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     }
     __syncwarp();
 
-    // producer (lane 0): slice pass pt, row pairs left in it, source and size of the next unit, ring slot
+    // producer (lane 0): slice pass pt, units left in it, source and unit size of the next copy, ring slot
     const uint32_t bars_a = smem_u32(bars), ring_a = smem_u32(ring);
     int pt = 0, pleft = 0, pslot = 0;
     uint32_t pbytes = 0;
     const unsigned char* psrc = codes;
     auto issue = [&]() {
         if (pt < n_sl) {
+            const int nun = min(RU, pleft);
+            const uint32_t bytes = (uint32_t)nun * pbytes;
             if (lane == 0) {
-                mbar_expect_tx(bars_a + 8 * pslot, pbytes);
-                bulk_copy_g2s(ring_a + pslot * kUnit2, psrc, pbytes, bars_a + 8 * pslot);
+                mbar_expect_tx(bars_a + 8 * pslot, bytes);
+                bulk_copy_g2s(ring_a + pslot * kSlot, psrc, bytes, bars_a + 8 * pslot);
             }
-            psrc += rp_stride;
-            if (--pleft == 0) {
+            psrc += bytes;
+            pleft -= nun;
+            if (pleft == 0) {
                 ++pt;
                 pleft = n_rp;
-                psrc = codes + (size_t)(sl_lane + pt * Wc) * kUnit2;
+                psrc = codes + unit_offset(L, rpw, min(sl_lane + pt * Wc, S - 1));
                 pbytes = (sl_lane + pt * Wc) == S - 1 ? (uint32_t)L.last_unit : (uint32_t)kUnit2;
             }
         }
@@ -232,7 +239,7 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
         }
         pt = n_rp > 0 ? 0 : n_sl;
         pleft = n_rp;
-        psrc = codes + (size_t)sl_lane * kUnit2;
+        psrc = codes + unit_offset(L, rpw, min(sl_lane, S - 1));
         pbytes = sl_lane == S - 1 ? (uint32_t)L.last_unit : (uint32_t)kUnit2;
         // x -> block fixed point in shared memory, two 16-column chunks per thread in flight.  Reads go to L2
         // (ld.global.cg), the point of coherence, never through L1.  The first reads are issued before the ring
@@ -290,13 +297,14 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
             // sum_j t_j X_j = sum_j q_j X_j - sum_j X_j: the low accumulators start at minus 4^f times the block sum;
             // the unmasked word stands for all four fields at once and starts at minus (1 + 4 + 16 + 64) times it
             const int n0 = -mt.y, n1 = -(mt.y << 2), n2 = -(mt.y << 4), n3 = -(mt.y * 85);
-            float* ppart = partial + (size_t)wi * 2 * S + sl + (lane >> 4) * S;
+            float* ppart = partial + (size_t)(2 * (rpw - rp0) + (lane >> 4)) * S + sl;
+            const int ubytes = sl == S - 1 ? L.last_unit : kUnit2;
             // a slot holds the unit as it lies in memory: atom (i, l) at 16 (i A + l), the scale quads after the atoms
             const int ln = live ? lane : 0;
             const int atom_stride = active * 16;
             const int scale_off = active * 64 + (ln >> 1) * 8 - ln * 16;
-            for (int j = 0; j < n_rp; ++j) {
-                // wait (bounded) for the unit in slot cslot; it has normally arrived long ago
+            for (int j0 = 0; j0 < n_rp; j0 += RU) {
+                // wait (bounded) for the copy in slot cslot; it has normally arrived long ago
                 if (!mbar_try_wait(bars_a + 8 * cslot, phase)) {
                     const int limit = failed ? kSpinLimitAfterFailure : kSpinLimit;
                     int spins = 0;
@@ -304,7 +312,10 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                         if (++spins >= limit) { failed = true; break; }
                     }
                 }
-                const unsigned char* buf = ring + cslot * kUnit2 + ln * 16;
+                const int nun = min(RU, n_rp - j0);
+                const unsigned char* buf = ring + cslot * kSlot + ln * 16;
+#pragma unroll 1
+                for (int u = 0; u < nun; ++u, buf += ubytes) {
                 // Fields 0..2 are masked out of each code word; the unmasked word gives the sum of all four fields
                 // (a byte is q0 + 4 q1 + 16 q2 + 64 q3 <= 170), so field 3 is "all" minus the other three.
                 int ah[4] = {0, 0, 0, 0};
@@ -335,17 +346,18 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                 // (their block scale c0 is zero and the unit they read is real data, so their products are zero)
                 float y0 = c0 * fmaf(0.25f, s0.y * (float)Q1, s0.x * (float)Q0);
                 float y1 = c1 * fmaf(0.25f, s1.y * (float)Q3, s1.x * (float)Q2);
-                // every lane has consumed the slot: lane 0 may refill it
-                __syncwarp();
-                issue();
-                if (++cslot == D) { cslot = 0; phase ^= 1u; }
                 // lanes 0-15 reduce row 0, lanes 16-31 row 1
                 const float send = (lane & 16) ? y0 : y1;
                 float v = ((lane & 16) ? y1 : y0) + __shfl_xor_sync(0xffffffffu, send, 16);
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
                 if ((lane & 15) == 0) *ppart = failed ? __int_as_float(0x7fc00000) : v;
-                ppart += (size_t)m * 2 * S;
+                ppart += 2 * S;
+                }
+                // every lane has consumed the slot: lane 0 may refill it
+                __syncwarp();
+                issue();
+                if (++cslot == D) { cslot = 0; phase ^= 1u; }
             }
         }
         if (!spec) break;
@@ -372,14 +384,14 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     }
 }
 
-size_t smem_bytes(const Layout2& L, int rows_cap, int warps, int depth, int speculate) {
-    return smem_layout2(L.k, L.slices, rows_cap, warps, depth, speculate).total;
+size_t smem_bytes(const Layout2& L, int rows_cap, int warps, int depth, int ru, int speculate) {
+    return smem_layout2(L.k, L.slices, rows_cap, warps, depth, ru, speculate).total;
 }
 
-template <int D>
+template <int D, int RU>
 ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int grid, int warps,
                       int rows_cap, size_t smem, int speculate, cudaStream_t st) {
-    auto kern = gemv2_kernel<D>;
+    auto kern = gemv2_kernel<D, RU>;
     static thread_local size_t configured[64] = {};       // per device: largest dynamic smem already allowed
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
@@ -436,17 +448,18 @@ ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st) {
 }
 
 // warps: per CTA, 0 = the default below, -1 = as many as fit (for a call that is known to run alone).
-// ctas_per_sm: CTAs of this launch per SM (0 = one).  The defaults keep a CTA small (4 to 8 warps, two ring slots
-// per warp) so that the CTAs of several consecutive launches are resident on an SM at once: under programmatic
-// dependent launch with speculative execution the head of one launch (fetching x) and the tail of another
-// (verifying x, reducing) then overlap the streaming of a third.  Measured on the LLaMA-3-8B shapes, 4 warps
-// beat 8 and 16 (6.9 / 7.3 / 8.5 us on 14336 x 4096).
+// ctas_per_sm: CTAs of this launch per SM (0 = one).  units: slice units per bulk copy (1, 2 or 4; 0 = 2).
+// The defaults keep a CTA small (4 to 8 warps, two ring slots of two units per warp) so that the CTAs of several
+// consecutive launches are resident on an SM at once: under programmatic dependent launch with speculative
+// execution the head of one launch (fetching x) and the tail of another (verifying x, reducing) then overlap the
+// streaming of a third.  Measured on the LLaMA-3-8B shapes, 4 warps beat 8 and 16.
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
-                          int ctas_per_sm, int depth, cudaStream_t st) {
+                          int ctas_per_sm, int depth, int units, cudaStream_t st) {
     const int S = L.slices;
     const int speculate = speculation_enabled() ? 1 : 0;
     if (ctas_per_sm < 0 || ctas_per_sm > 4) return PTQTP_ERR_CONFIG;
     if (warps < -1 || warps > kMaxWarps2) return PTQTP_ERR_CONFIG;
+    if (units != 0 && units != 1 && units != 2 && units != 4) return PTQTP_ERR_CONFIG;
     const int per_sm = ctas_per_sm ? ctas_per_sm : 1;
     const int max_warps = kMaxWarps2 / per_sm;
     const size_t budget = (size_t)(228 / per_sm - 1) * 1024;          // 228 KB per SM, 1 KB of it reserved per CTA
@@ -466,15 +479,29 @@ ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* 
     if (warps < 1 || warps > max_warps) return PTQTP_ERR_CONFIG;
     const int rows_cap = 2 * ((L.nrp + grid - 1) / grid);
     if (depth == 0) depth = 2;
-    const size_t smem = smem_bytes(L, rows_cap, warps, depth, speculate);
-    if (smem > budget) return depth > 2 || warps > 1 || ctas_per_sm == 2 ? PTQTP_ERR_CONFIG : PTQTP_ERR_SHAPE;
-    switch (depth) {
-        case 2: return launch_d<2>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
-        case 3: return launch_d<3>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
-        case 4: return launch_d<4>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
-        case 6: return launch_d<6>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
-        case 8: return launch_d<8>(L, packed, x, y, grid, warps, rows_cap, smem, speculate, st);
+    int spec = speculate;
+    if (units == 0) {
+        // two units per copy; for long K one, and then without the second copy of x that speculative execution keeps
+        // (two only while three such CTAs still fit on an SM: sharing the SM with the neighbouring launches is
+        // worth more than cheaper copies)
+        units = smem_bytes(L, rows_cap, warps, depth, 2, spec) <= min(budget, (size_t)75 * 1024) ? 2 : 1;
+        if (smem_bytes(L, rows_cap, warps, depth, units, spec) > budget) spec = 0;
     }
+    const size_t smem = smem_bytes(L, rows_cap, warps, depth, units, spec);
+    if (smem > budget) return depth > 2 || warps > 1 || units > 1 || ctas_per_sm == 2 ? PTQTP_ERR_CONFIG : PTQTP_ERR_SHAPE;
+#define PTQTP_LAUNCH_D(DD)                                                                                            \
+    case DD:                                                                                                          \
+        return units == 1 ? launch_d<DD, 1>(L, packed, x, y, grid, warps, rows_cap, smem, spec, st)                   \
+             : units == 2 ? launch_d<DD, 2>(L, packed, x, y, grid, warps, rows_cap, smem, spec, st)                   \
+                          : launch_d<DD, 4>(L, packed, x, y, grid, warps, rows_cap, smem, spec, st);
+    switch (depth) {
+        PTQTP_LAUNCH_D(2)
+        PTQTP_LAUNCH_D(3)
+        PTQTP_LAUNCH_D(4)
+        PTQTP_LAUNCH_D(6)
+        PTQTP_LAUNCH_D(8)
+    }
+#undef PTQTP_LAUNCH_D
     return PTQTP_ERR_CONFIG;
 }
 

@@ -232,7 +232,7 @@ gemv3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                     const uint32_t bytes = ps == S - 1 ? (uint32_t)L.last_unit : (uint32_t)kUnit2;
                     bar_expect_tx(full + pstage, bytes);
                     bulk_g2s(ring + pstage * kStage3 + hq * kUnitStride3,
-                             codes + (size_t)(4 * q + hq) * L.strip + (size_t)ps * kUnit2, bytes, full + pstage);
+                             codes + unit_offset(L, 4 * q + hq, ps), bytes, full + pstage);
                 } else {
                     bar_arrive(full + pstage);          // a row pair past the end of the matrix: nothing to bring
                 }

@@ -27,7 +27,7 @@ __device__ __forceinline__ Atom atom_of(const Layout2& L, size_t a) {
     t.active = active_of(L, t.slice);
     t.i = r / t.active;
     t.lane = r % t.active;
-    t.unit_off = (size_t)t.rp * L.strip + (size_t)t.slice * kUnit2;
+    t.unit_off = unit_offset(L, t.rp, t.slice);
     return t;
 }
 
@@ -94,7 +94,7 @@ __global__ void pack2_kernel(Layout2 L, const int8_t* __restrict__ T1, const int
                 s[2 * r + 1] = a2[(size_t)row * groups + g];
             }
         }
-        unsigned char* dst = codes + (size_t)rp * L.strip + (size_t)slice * kUnit2 + (size_t)active * 64 + gl * 8;
+        unsigned char* dst = codes + unit_offset(L, rp, slice) + (size_t)active * 64 + gl * 8;
         *reinterpret_cast<uint2*>(dst) = make_uint2((uint32_t)s[0] | ((uint32_t)s[1] << 16),
                                                     (uint32_t)s[2] | ((uint32_t)s[3] << 16));
     }
@@ -103,7 +103,7 @@ __global__ void pack2_kernel(Layout2 L, const int8_t* __restrict__ T1, const int
     const int last_content = L.last_active * 64 + L.last_active * 4;
     if (last_content < L.last_unit) {
         for (size_t rp = tid; rp < (size_t)L.nrp; rp += stride) {
-            unsigned char* dst = codes + rp * L.strip + (size_t)(L.slices - 1) * kUnit2;
+            unsigned char* dst = codes + unit_offset(L, (int)rp, L.slices - 1);
             for (int b = last_content; b < L.last_unit; ++b) dst[b] = 0;
         }
     }
@@ -170,7 +170,7 @@ __global__ void unpack2_kernel(Layout2 L, const unsigned char* __restrict__ pack
         const int rp = (int)(q / groups), g = (int)(q % groups);
         const int slice = g / 16, gl = g % 16;
         const int active = active_of(L, slice);
-        const uint2 s = *reinterpret_cast<const uint2*>(codes + (size_t)rp * L.strip + (size_t)slice * kUnit2 +
+        const uint2 s = *reinterpret_cast<const uint2*>(codes + unit_offset(L, rp, slice) +
                                                         (size_t)active * 64 + gl * 8);
         const uint32_t v[2] = {s.x, s.y};
 #pragma unroll

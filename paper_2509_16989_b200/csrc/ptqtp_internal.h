@@ -56,7 +56,7 @@ struct Layout2 {
     int slices;                      // ceil(k / 2048)
     int last_active;                 // 64-column lane blocks in the last slice (1..32)
     int last_unit;                   // bytes of the last slice's unit (multiple of 16)
-    size_t strip;                    // bytes of one row pair: (slices - 1) * 2176 + last_unit
+    size_t strip;                    // bytes of one row pair over all slices: (slices - 1) * 2176 + last_unit
     size_t codes_off, total;
 };
 
@@ -73,6 +73,12 @@ inline Layout2 make_layout2(const ptqtp_shape* s) {
     L.codes_off = PTQTP_HEADER_BYTES;
     L.total = L.codes_off + (size_t)L.nrp * L.strip;
     return L;
+}
+
+// Byte offset (from codes_off) of the slice unit of row pair rp and slice s.  Slice-major: all units of slice 0,
+// then all units of slice 1, ...; the units of one slice for consecutive row pairs are contiguous.
+__host__ __device__ inline size_t unit_offset(const Layout2& L, int rp, int s) {
+    return (size_t)s * L.nrp * kUnit2 + (size_t)rp * (s == L.slices - 1 ? L.last_unit : kUnit2);
 }
 
 inline size_t packed_total(const ptqtp_shape* s) {
@@ -98,7 +104,7 @@ ptqtp_status launch_pack2(const Layout2& L, const int8_t* T1, const int8_t* T2, 
 ptqtp_status launch_unpack2(const Layout2& L, const void* packed, int8_t* T1, int8_t* T2, uint16_t* a1,
                             uint16_t* a2, int32_t* dev_status, cudaStream_t st);
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
-                          int ctas_per_sm, int depth, cudaStream_t st);
+                          int ctas_per_sm, int depth, int units, cudaStream_t st);
 ptqtp_status launch_skinny2(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y,
                             cudaStream_t st);
 size_t skinny3_workspace_bytes(int k, int m);

@@ -164,7 +164,7 @@ skinny2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half
 #pragma unroll
             for (int uu = 0; uu < 4; ++uu) {
                 const int rp = min(4 * q + uu, L.nrp - 1);                     // row pairs past the end re-read the last one
-                const unsigned char* src = codes + (size_t)rp * L.strip + (size_t)sl * kUnit2;
+                const unsigned char* src = codes + unit_offset(L, rp, sl);
                 unsigned char* d = dst + uu * (kSU * 16);
                 if (ll < Ah) {
                     cp16(d + (ip * kSI + ll) * 16, src + (ip * A + l0 + ll) * 16);

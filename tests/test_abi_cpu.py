@@ -57,7 +57,7 @@ def test_parse_header_accepts_reference_blob_and_rejects_damage(L):
     blob2 = pf.pack_reference_v2(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
     assert binding.ptqtp_parse_header(bytes(blob2[:256])) == (3, 1152, 2)
     bad2 = blob2[:256].copy()
-    bad2[40] ^= 8         # row-pair stride no longer matches the shape
+    bad2[40] ^= 8         # bytes per row pair no longer match the shape
     with pytest.raises(binding.PtqtpError):
         binding.ptqtp_parse_header(bytes(bad2))
     blob = pf.pack_reference(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
@@ -123,24 +123,26 @@ def test_reference_format2_roundtrip_layout_and_damage_detection():
     assert np.array_equal(t1, c["T1"]) and np.array_equal(t2, c["T2"])
     assert np.array_equal(a1.view(np.uint16), c["alpha1"].view(np.uint16))
     assert np.array_equal(a2.view(np.uint16), c["alpha2"].view(np.uint16))
-    # one byte by hand: row pair 1 (rows 2, 3), column 2048 + 64*3 + 16*2 + 5 = 2277:
-    # slice 1, lane block 3, sub-block 2, byte 5 -> strip offset 2176 + 16 * (2 * 32 + 3) + 5
-    strip = 2 * 2176 + 144
-    off = 256 + 1 * strip + 2176 + 16 * (2 * 32 + 3) + 5
+    # the body is slice-major: 3 row pairs x 2176 bytes of slice 0, 3 x 2176 of slice 1, 3 x 144 of the tail slice.
+    # One byte by hand: row pair 1 (rows 2, 3), column 2048 + 64*3 + 16*2 + 5 = 2277:
+    # slice 1, lane block 3, sub-block 2, byte 5 -> unit offset 16 * (2 * 32 + 3) + 5
+    run = 3 * 2176
+    off = 256 + run + 1 * 2176 + 16 * (2 * 32 + 3) + 5
     want = ((int(c["T1"][2, 2277]) + 1) | (int(c["T2"][2, 2277]) + 1) << 2 | (int(c["T1"][3, 2277]) + 1) << 4
             | (int(c["T2"][3, 2277]) + 1) << 6)
     assert int(blob[off]) == want
     # scale quad of row pair 0, group 17 (slice 1, second group): after the 2048 code bytes of that unit
-    q = 256 + 2176 + 2048 + 8 * 1
+    q = 256 + run + 2048 + 8 * 1
     assert bytes(blob[q:q + 8]) == (c["alpha1"][0, 17].tobytes() + c["alpha2"][0, 17].tobytes()
                                     + c["alpha1"][1, 17].tobytes() + c["alpha2"][1, 17].tobytes())
-    # the tail unit: 128 columns -> 2 lane blocks, 128 code bytes, one quad, 8 bytes of zero padding
-    tail = 256 + 2 * 2176
+    # the tail unit of row pair 0: 128 columns -> 2 lane blocks, 128 code bytes, one quad, 8 bytes of zero padding
+    tail = 256 + 2 * run
     assert bytes(blob[tail + 128:tail + 136]) == (c["alpha1"][0, 32].tobytes() + c["alpha2"][0, 32].tobytes()
                                                   + c["alpha1"][1, 32].tobytes() + c["alpha2"][1, 32].tobytes())
     assert not blob[tail + 136:tail + 144].any()
-    # the missing row 5 is trit 0 (code 1) with zero scales
-    last = 256 + 2 * strip
+    assert blob.size == 256 + 2 * run + 3 * 144
+    # the missing row 5 is trit 0 (code 1) with zero scales: first byte of row pair 2 in slice 0
+    last = 256 + 2 * 2176
     assert (int(blob[last]) >> 4) == 0b0101
     bad = blob.copy()
     bad[256] |= 3

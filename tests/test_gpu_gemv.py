@@ -46,13 +46,17 @@ def test_format2_launch_configurations(warps, depth):
         ref = oracle_y(c)
         packed = pack_case(c, binding.FORMAT_V2)
         # shared memory: x as two byte planes + block records, the first read of x (speculative execution is on
-        # by default), the slice partials, one mbarrier and one 2176-byte slot per ring entry
+        # by default), the slice partials, one mbarrier and one slot of two 2176-byte units per ring entry
         S = -(-K // 2048)
         nrp = (N + 1) // 2
         rows_cap = 2 * -(-nrp // min(148, nrp))
         raw_off = -(-((K // 64) * 136) // 16) * 16
         bar_off = -(-(raw_off + 2 * K + rows_cap * S * 4) // 8) * 8
-        smem = -(-(bar_off + warps * depth * 8) // 16) * 16 + warps * depth * 2176
+        smem = -(-(bar_off + warps * depth * 8) // 16) * 16 + warps * depth * 2 * 2176
+        if smem > 75 * 1024:                             # the library falls back to one unit per copy
+            smem -= warps * depth * 2176
+        if smem > 227 * 1024:                            # ... and then does without the first read of x
+            smem -= 2 * K
         if smem > 227 * 1024:
             with pytest.raises(binding.PtqtpError) as e:
                 binding.ptqtp_gemv_cfg(packed, N, K, dev(c["x"]), k_split=warps, depth=depth, fmt=binding.FORMAT_V2)
@@ -63,15 +67,48 @@ def test_format2_launch_configurations(warps, depth):
         assert_parity(y.cpu().numpy(), ref, c["x"], "warps=%d depth=%d N=%d K=%d" % (warps, depth, N, K))
 
 
+def _cuda_core_config_fits(N, K, warps, depth, units, per_sm):
+    """Host-side model of the CUDA-core kernel's launch rules: does this configuration fit in shared memory?"""
+    S, nrp, p = -(-K // 2048), (N + 1) // 2, per_sm or 1
+    max_warps, grid = 16 // p, min(p * 148, nrp)
+    if warps == 0:
+        target = 8 if -(-nrp // grid) * S >= 256 else 4
+        warps = max_warps if S >= max_warps else S * -(-target // S)
+        if warps > max_warps:
+            warps = S * (max_warps // S)
+    if warps < 1 or warps > max_warps:
+        return False
+    rows_cap, depth = 2 * -(-nrp // grid), depth or 2
+
+    def smem(u, spec):
+        raw_off = -(-((K // 64) * 136) // 16) * 16
+        bar_off = -(-(raw_off + (2 * K if spec else 0) + rows_cap * S * 4) // 8) * 8
+        return -(-(bar_off + warps * depth * 8) // 16) * 16 + warps * depth * u * 2176
+
+    budget = (228 // p - 1) * 1024
+    if units == 0:                                       # the library's own fallbacks
+        u = 2 if smem(2, 1) <= min(budget, 75 * 1024) else 1
+        return smem(u, 1) <= budget or smem(u, 0) <= budget
+    return smem(units, 1) <= budget
+
+
 @pytest.mark.parametrize("per_sm", [0, 1, 2])
+@pytest.mark.parametrize("units", [0, 1, 2, 4])
 @pytest.mark.parametrize("warps,depth", [(0, 0), (4, 2), (8, 3), (7, 2), (2, 4)])
-def test_format2_ctas_per_sm(warps, depth, per_sm):
-    for N, K in ((300, 4096), (1000, 14336), (5, 2048), (2400, 1024), (4097, 6144)):
+def test_format2_ctas_per_sm_and_units_per_copy(warps, depth, units, per_sm):
+    # rows_per_warp is, for format 2, the number of slice units one bulk copy brings
+    for N, K in ((300, 4096), (1000, 14336), (5, 2048), (2400, 1024), (4097, 6144), (23, 128)):
         c = make_case(N, K, seed=warps + depth)
-        y = binding.ptqtp_gemv_cfg(pack_case(c, binding.FORMAT_V2), N, K, dev(c["x"]), k_split=warps, depth=depth,
-                                   ctas_per_sm=per_sm, fmt=binding.FORMAT_V2)
+        cfg = dict(rows_per_warp=units, k_split=warps, depth=depth, ctas_per_sm=per_sm, fmt=binding.FORMAT_V2)
+        if not _cuda_core_config_fits(N, K, warps, depth, units, per_sm):
+            with pytest.raises(binding.PtqtpError) as e:
+                binding.ptqtp_gemv_cfg(pack_case(c, binding.FORMAT_V2), N, K, dev(c["x"]), **cfg)
+            assert e.value.status == binding.ERR_CONFIG
+            continue
+        y = binding.ptqtp_gemv_cfg(pack_case(c, binding.FORMAT_V2), N, K, dev(c["x"]), **cfg)
         torch.cuda.synchronize()
-        assert_parity(y.cpu().numpy(), oracle_y(c), c["x"], "warps=%d depth=%d per_sm=%d N=%d K=%d" % (warps, depth, per_sm, N, K))
+        assert_parity(y.cpu().numpy(), oracle_y(c), c["x"],
+                      "warps=%d depth=%d units=%d per_sm=%d N=%d K=%d" % (warps, depth, units, per_sm, N, K))
 
 
 @pytest.mark.parametrize("arith", [3, 4])
@@ -133,7 +170,7 @@ def test_format2_tensor_core_kernel_is_exact_on_integers():
 def test_format2_rejects_format1_only_options():
     c = make_case(8, 1024, seed=1)
     packed = pack_case(c, binding.FORMAT_V2)
-    for bad in (dict(rows_per_warp=2), dict(arith=1), dict(k_split=17), dict(depth=5),
+    for bad in (dict(rows_per_warp=3), dict(rows_per_warp=8), dict(arith=4, rows_per_warp=2), dict(arith=1), dict(k_split=17), dict(depth=5),
                 dict(arith=4, k_split=7), dict(arith=4, depth=9), dict(arith=4, depth=1), dict(arith=4, ctas_per_sm=3),
                 dict(ctas_per_sm=5)):
         with pytest.raises(binding.PtqtpError) as e:
