@@ -199,13 +199,14 @@ PTQTP_API ptqtp_status ptqtp_gemv_host(const ptqtp_shape *shape /* host */, cons
  * arith: accumulation of the sign-selected activations -- 0 = fp32 accumulator fed by mixed-precision
  * FMAs (fp16 operands), 1 = fp16x2 chains of 4 flushed into fp32, 2 = chains of 8, -1 = library choice.
  * PTQTP_ERR_CONFIG if the combination is not built.
- * For a format-2 blob the arguments mean: rows_per_warp must be 0; arith = -1 (library choice), 3 (masks and
- * integer dot products on the CUDA cores) or 4 (int8 tensor-core MMAs, the kernel behind ptqtp_gemm_skinny for
- * two to four rows).  arith 3: k_split = warps per CTA (1..16 / ctas_per_sm, 0 = auto: 4 to 8, so that the CTAs
- * of several consecutive launches fit on an SM together; 16 serves a call that runs alone best);
- * ctas_per_sm = CTAs of this launch per SM (1..4, 0 = 1); depth = slice units in flight per warp (2, 3, 4, 6,
- * 8; 0 = 2).  arith 4: k_split = warps per CTA (4, 8 or 16, 0 = auto); ctas_per_sm 1 or 2 (0 = 1); depth =
- * stages (four slice units each) per team of four warps (2..8, 0 = auto). */
+ * For a format-2 blob the arguments mean: arith = -1 (library choice), 3 (masks and integer dot products on
+ * the CUDA cores) or 4 (int8 tensor-core MMAs, the kernel behind ptqtp_gemm_skinny for two to four rows).
+ * arith 3: rows_per_warp = slice units per bulk copy (1, 2 or 4; 0 = 2, or 1 when x is long); k_split = warps
+ * per CTA (1..16 / ctas_per_sm, 0 = auto: 4 to 8, so that the CTAs of several consecutive launches fit on an SM
+ * together; 16 serves a call that runs alone best); ctas_per_sm = CTAs of this launch per SM (1..4, 0 = 1);
+ * depth = copies in flight per warp (2, 3, 4, 6, 8; 0 = 2).  arith 4: rows_per_warp must be 0; k_split = warps
+ * per CTA (4, 8 or 16, 0 = auto); ctas_per_sm 1 or 2 (0 = 1); depth = stages (four slice units each) per team of
+ * four warps (2..8, 0 = auto).  A configuration that does not fit in shared memory gives PTQTP_ERR_CONFIG. */
 PTQTP_API ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                             const uint16_t *x, uint16_t *y, int32_t rows_per_warp, int32_t k_split,
                             int32_t ctas_per_sm, int32_t depth, int32_t arith, void *stream);
