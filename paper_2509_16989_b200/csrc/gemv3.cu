@@ -79,6 +79,7 @@ __device__ __forceinline__ bool bar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // returns false when the wait gave up
 __device__ __forceinline__ bool bar_wait_bounded(uint64_t* bar, uint32_t parity, bool already_failed) {
+    if (bar_try_wait(bar, parity)) return true;         // what is waited for has normally happened long ago
     const int limit = already_failed ? kSpinAfterFailure3 : kSpin3;
     int spins = 0;
     while (!bar_try_wait(bar, parity)) {
@@ -190,7 +191,8 @@ gemv3_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     float* partial = reinterpret_cast<float*>(smem + sm.partial_off);       // [m][rows_cap][S kTeamWarps]
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bar_off);        // per team: depth "full", depth "empty"
     unsigned char* rings = smem + sm.ring_off;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // (the shuffle tells the compiler that the warp index is the same in all lanes)
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const int cthreads = teams * kTeamWarps * 32;
     const int team = warp / kTeamWarps, hq = warp % kTeamWarps, g = lane >> 2, t = lane & 3;
     uint64_t* full = bars + team * 2 * depth;
