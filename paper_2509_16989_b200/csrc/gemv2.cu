@@ -472,7 +472,7 @@ ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* 
         // a multiple of the slice count (every slice lane gets as many warps): at least 4, at least 8 when a CTA
         // streams many units, and all 16 when that is what it takes to give every slice a warp
         const long units_per_cta = (long)((L.nrp + grid - 1) / grid) * S;
-        const int target = units_per_cta >= 256 ? 8 : 4;
+        const int target = units_per_cta >= 160 ? 8 : 4;  // (a long launch with 4 warps holds up the short ones behind it)
         warps = S >= max_warps ? max_warps : S * ((target + S - 1) / S);
         if (warps > max_warps) warps = S * (max_warps / S);
     }

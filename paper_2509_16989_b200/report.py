@@ -5,6 +5,9 @@
   0  Qwen3-0.6B up_proj 3072 x 1024, batch 1
   2  batch sweep M in {1,...,64} of ptqtp_gemm_skinny on the 14336 x 4096 gate/up shape (and ptqtp_gemv at M = 1)
   3  LLaMA-3-70B shapes, planes with P(0) = 0.5, batch 1 and 8
+  5  a LLaMA-3-8B layer with stacked matrices: q, k, v packed as one 6144 x 4096 matrix, and also gate, up as one
+     28672 x 4096 matrix (rows are independent, so a caller may stack matrices that share their input and
+     slice y): five or four calls per layer instead of seven
 
 (The 32-layer stack built from decomposed weights needs the CPU oracle to prepare its inputs and is therefore
 measured by tests/test_gpu_stack.py.)
@@ -132,9 +135,39 @@ def config3(T):
         torch.cuda.empty_cache()
 
 
+def config5(T):
+    # the chain walks over enough copies of the layer to exceed twice the L2 size
+    variants = [
+        ("stacked q/k/v", [("qkv", 6144, 4096), ("o", 4096, 4096), ("gate", 14336, 4096), ("up", 14336, 4096),
+                           ("down", 4096, 14336)]),
+        ("stacked q/k/v and gate/up", [("qkv", 6144, 4096), ("o", 4096, 4096), ("gate_up", 28672, 4096),
+                                       ("down", 4096, 14336)]),
+    ]
+    for what, shapes in variants:
+        base = {}
+        for i, (name, N, K) in enumerate(shapes):
+            c = make_case(N, K, seed=50 + i)
+            packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
+            base[name] = (packed, dev(c["x"]), torch.empty(N, dtype=torch.float16, device="cuda"))
+        layer_bytes = sum(base[n][0].numel() for n, _, _ in shapes)
+        copies = max(4, -(-(2 * T.l2 + (64 << 20)) // layer_bytes))
+        layers = [{n: (base[n][0] if l == 0 else base[n][0].clone()) for n, _, _ in shapes} for l in range(copies)]
+        calls = []
+        for l in range(copies):
+            for name, N, K in shapes:
+                calls.append(lambda p=layers[l][name], N=N, K=K, x=base[name][1], y=base[name][2]:
+                             binding.ptqtp_gemv(p, N, K, x, y=y, stream=T.stream))
+        us = T.steady_us(calls) * len(shapes)
+        nb = sum(algorithmic_bytes(N, K) for _, N, K in shapes)
+        emit(workload="cfg5 llama3-8b layer, " + what, call="%d x ptqtp_gemv" % len(shapes), us_per_layer=round(us, 3),
+             gbs=round(nb / us / 1e3, 1), bytes=nb, layer_copies=copies)
+        del layers, base, calls
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="0,2,3")
+    ap.add_argument("--only", default="0,2,3,5")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise RuntimeError("needs a CUDA device")
@@ -147,6 +180,8 @@ def main():
         config2(T)
     if 3 in which:
         config3(T)
+    if 5 in which:
+        config5(T)
 
 
 if __name__ == "__main__":

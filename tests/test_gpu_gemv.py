@@ -72,7 +72,7 @@ def _cuda_core_config_fits(N, K, warps, depth, units, per_sm):
     S, nrp, p = -(-K // 2048), (N + 1) // 2, per_sm or 1
     max_warps, grid = 16 // p, min(p * 148, nrp)
     if warps == 0:
-        target = 8 if -(-nrp // grid) * S >= 256 else 4
+        target = 8 if -(-nrp // grid) * S >= 160 else 4
         warps = max_warps if S >= max_warps else S * -(-target // S)
         if warps > max_warps:
             warps = S * (max_warps // S)
@@ -165,6 +165,18 @@ def test_format2_tensor_core_kernel_is_exact_on_integers():
     for arith in (3, 4):
         y = run_gemv(c, binding.FORMAT_V2, arith=arith)
         assert np.array_equal(y.astype(np.float64), ref.astype(np.float16).astype(np.float64)), arith
+
+
+def test_stacked_matrices_give_the_rows_of_separate_calls():
+    # rows are independent: packing [W1; W2] as one matrix and slicing y is the same computation, bit for bit
+    K = 4096
+    c1, c2 = make_case(1024, K, seed=71), make_case(300, K, seed=72)
+    c2["x"] = c1["x"]
+    stacked = dict(N=1324, K=K, x=c1["x"], **{k: np.concatenate([c1[k], c2[k]]) for k in ("T1", "T2", "alpha1", "alpha2")})
+    y1, y2, ys = run_gemv(c1, binding.FORMAT_V2), run_gemv(c2, binding.FORMAT_V2), run_gemv(stacked, binding.FORMAT_V2)
+    assert np.array_equal(ys[:1024].view(np.uint16), y1.view(np.uint16))
+    assert np.array_equal(ys[1024:].view(np.uint16), y2.view(np.uint16))
+    assert_parity(ys, oracle_y(stacked), stacked["x"], "stacked")
 
 
 def test_format2_rejects_format1_only_options():
