@@ -106,3 +106,21 @@ def parity_metrics(y_test, y_ref, x):
         bound = 2e-3 * float(np.max(np.abs(X[m]))) * np.sqrt(X.shape[1]) if X.shape[1] else 0.0
         out.append((float(rel), mab, bound))
     return out
+
+
+def swiglu_fp64(T1, T2, alpha1, alpha2, x, G=128):
+    """Gated pair epilogue on top of the layer product, fp64 (batch 1 or [M, K]).
+
+    The matrix holds gate and up projections interleaved by rows: row 2i is gate row i, row 2i+1 is up row i
+    (the MLP of the LLaMA / Qwen models the paper quantises computes down(silu(gate(x)) * up(x)); the paper's
+    layer, Eq. 1-2, is what produces gate(x) and up(x)).  With t = layer_fp64(...):
+
+        y[i] = silu(t[2i]) * t[2i+1],     silu(g) = g / (1 + exp(-g))
+
+    Returns [N/2] or [M, N/2].
+    """
+    t = layer_fp64(T1, T2, alpha1, alpha2, x, G)
+    if t.shape[-1] % 2:
+        raise ValueError("an even number of rows is required (gate and up rows come in pairs)")
+    g, u = t[..., 0::2], t[..., 1::2]
+    return g / (1.0 + np.exp(-g)) * u
