@@ -139,6 +139,16 @@ PTQTP_API ptqtp_status ptqtp_unpack(const ptqtp_shape *shape /* host */, const v
 PTQTP_API ptqtp_status ptqtp_gemv(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                         const uint16_t *x, uint16_t *y, void *stream);
 
+/* ptqtp_gemv with a gated pair epilogue, for the MLP of the LLaMA / Qwen models the paper quantises
+ * (down(silu(gate(x)) * up(x)); the paper's layer, Eq. 1-2, is what yields gate(x) and up(x)).  The caller packs
+ * ONE matrix of N rows (N even) that holds the gate and up projections interleaved by rows: row 2i = gate row i,
+ * row 2i+1 = up row i.  With t = the layer's N fp32 row sums (before any rounding to fp16),
+ *     y[i] = silu(t[2i]) * t[2i+1],   silu(g) = g / (1 + exp(-g)),   i < N/2,
+ * rounded once to fp16.  y: device fp16 [N/2].  Format 2 only (PTQTP_ERR_CONFIG for format 1); PTQTP_ERR_SHAPE for
+ * odd N.  Everything else as ptqtp_gemv (same kernel: only its final store differs). */
+PTQTP_API ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
+                               const uint16_t *x, uint16_t *y, void *stream);
+
 /* Small-batch variant: Y[m,:] = layer(X[m,:]) for m < M, 1 <= M <= PTQTP_MAX_BATCH.
  * X: device fp16 [M*K] row-major; Y: device fp16 [M*N] row-major.  Same definition per row of X.
  * Format 2, M >= 2: the planes are contracted on the tensor cores with int8 warp MMAs against 15-bit

@@ -24,7 +24,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_SIZE, ERR_TRIT, ERR_FORMAT, ERR_CUDA, ER
 EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny",
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
            "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws",
-           "ptqtp_gemm_skinny_static", "ptqtp_kernel_status")
+           "ptqtp_gemm_skinny_static", "ptqtp_kernel_status", "ptqtp_gemv_swiglu")
 
 
 class PtqtpError(RuntimeError):
@@ -60,6 +60,8 @@ def lib():
         L.ptqtp_unpack.argtypes = [sp, vp, sz, vp, vp, vp, vp, vp, vp]
         L.ptqtp_gemv.restype = ctypes.c_int
         L.ptqtp_gemv.argtypes = [sp, vp, sz, vp, vp, vp]
+        L.ptqtp_gemv_swiglu.restype = ctypes.c_int
+        L.ptqtp_gemv_swiglu.argtypes = [sp, vp, sz, vp, vp, vp]
         L.ptqtp_gemm_skinny.restype = ctypes.c_int
         L.ptqtp_gemm_skinny.argtypes = [sp, vp, sz, i32, vp, vp, vp]
         L.ptqtp_gemm_skinny_workspace_size.restype = sz
@@ -175,6 +177,17 @@ def ptqtp_gemv_cfg(packed, N, K, x, y=None, rows_per_warp=0, k_split=0, ctas_per
                               int(rows_per_warp), int(k_split), int(ctas_per_sm), int(depth), int(arith),
                               _stream_ptr(stream))
     _check(st, "ptqtp_gemv_cfg")
+    return y
+
+
+def ptqtp_gemv_swiglu(packed, N, K, x, y=None, stream=None):
+    """y[N/2] = silu(row 2i) * row 2i+1 of the layer applied to x; packed holds gate/up rows interleaved (format 2)."""
+    shape = make_shape(N, K, fmt=FORMAT_V2)
+    if y is None:
+        y = torch.empty(N // 2, dtype=torch.float16, device=x.device)
+    st = lib().ptqtp_gemv_swiglu(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
+                                 _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"), _stream_ptr(stream))
+    _check(st, "ptqtp_gemv_swiglu")
     return y
 
 

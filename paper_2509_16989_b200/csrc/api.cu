@@ -128,6 +128,18 @@ ptqtp_status ptqtp_gemv(const ptqtp_shape* shape, const void* packed, size_t pac
     return ptqtp_gemv_cfg(shape, packed, packed_bytes, x, y, 0, 0, 0, 0, -1, stream);
 }
 
+ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, const uint16_t* x,
+                               uint16_t* y, void* stream) {
+    if (!x || !y) return PTQTP_ERR_NULL;
+    AnyLayout L;
+    ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
+    if (s != PTQTP_OK) return s;
+    if (!L.v2) return PTQTP_ERR_CONFIG;
+    if (shape->n_out % 2) return PTQTP_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(y)) return PTQTP_ERR_ALIGN;
+    return launch_gemv2(L.l2, packed, x, y, 0, 0, 0, 0, static_cast<cudaStream_t>(stream), true);
+}
+
 ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, int32_t m,
                                const uint16_t* X, uint16_t* Y, void* stream) {
     if (!X || !Y) return PTQTP_ERR_NULL;

@@ -158,7 +158,7 @@ __host__ __device__ inline Smem2 smem_layout2(int k, int slices, int rows_cap, i
 template <int D, int RU>
 __global__ void __launch_bounds__(kMaxThreads2, 1)
 gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
-             __half* __restrict__ y, int rows_cap, int rp_base, int rp_rem, int speculate) {
+             __half* __restrict__ y, int rows_cap, int rp_base, int rp_rem, int speculate, int gated) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int nblk = L.k / kLane2;
     uint32_t* xhi = reinterpret_cast<uint32_t*>(smem);
@@ -375,6 +375,19 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
     }
     if (failed && lane == 0) atomicExch(&g_gemv2_status, (int)PTQTP_ERR_CUDA);
     __syncthreads();
+    if (gated) {
+        // gated pair epilogue: a row pair is (gate row, up row) and gives one output silu(gate) * up, computed
+        // from the unrounded fp32 sums
+        for (int r = threadIdx.x; r < rp1 - rp0; r += blockDim.x) {
+            float g = 0.f, u = 0.f;
+            for (int s = 0; s < S; ++s) {
+                g += partial[(size_t)(2 * r) * S + s];
+                u += partial[(size_t)(2 * r + 1) * S + s];
+            }
+            y[rp0 + r] = __float2half_rn(g / (1.f + expf(-g)) * u);
+        }
+        return;
+    }
     const int rows = 2 * (rp1 - rp0);
     for (int r = threadIdx.x; r < rows; r += blockDim.x) {
         const int row = 2 * rp0 + r;
@@ -390,7 +403,7 @@ size_t smem_bytes(const Layout2& L, int rows_cap, int warps, int depth, int ru, 
 
 template <int D, int RU>
 ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int grid, int warps,
-                      int rows_cap, size_t smem, int speculate, cudaStream_t st) {
+                      int rows_cap, size_t smem, int speculate, int gated, cudaStream_t st) {
     auto kern = gemv2_kernel<D, RU>;
     static thread_local size_t configured[64] = {};       // per device: largest dynamic smem already allowed
     int dev = 0;
@@ -419,7 +432,7 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
     cfg.numAttrs = overlap_enabled() ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, L, static_cast<const unsigned char*>(packed),
                                        reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap,
-                                       L.nrp / grid, L.nrp % grid, speculate);
+                                       L.nrp / grid, L.nrp % grid, speculate, gated);
     if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
     return PTQTP_OK;
 }
@@ -447,6 +460,7 @@ ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st) {
     return PTQTP_OK;
 }
 
+// gated: y[i] = silu(row 2i) * row 2i+1 instead of the rows themselves (N even).
 // warps: per CTA, 0 = the default below, -1 = as many as fit (for a call that is known to run alone).
 // ctas_per_sm: CTAs of this launch per SM (0 = one).  units: slice units per bulk copy (1, 2 or 4; 0 = 2).
 // The defaults keep a CTA small (4 to 8 warps, two ring slots of two units per warp) so that the CTAs of several
@@ -454,7 +468,7 @@ ptqtp_status copy_gemv2_status(int32_t* status_host, cudaStream_t st) {
 // execution the head of one launch (fetching x) and the tail of another (verifying x, reducing) then overlap the
 // streaming of a third.  Measured on the LLaMA-3-8B shapes, 4 warps beat 8 and 16.
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
-                          int ctas_per_sm, int depth, int units, cudaStream_t st) {
+                          int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated) {
     const int S = L.slices;
     const int speculate = speculation_enabled() ? 1 : 0;
     if (ctas_per_sm < 0 || ctas_per_sm > 4) return PTQTP_ERR_CONFIG;
@@ -491,9 +505,9 @@ ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* 
     if (smem > budget) return depth > 2 || warps > 1 || units > 1 || ctas_per_sm == 2 ? PTQTP_ERR_CONFIG : PTQTP_ERR_SHAPE;
 #define PTQTP_LAUNCH_D(DD)                                                                                            \
     case DD:                                                                                                          \
-        return units == 1 ? launch_d<DD, 1>(L, packed, x, y, grid, warps, rows_cap, smem, spec, st)                   \
-             : units == 2 ? launch_d<DD, 2>(L, packed, x, y, grid, warps, rows_cap, smem, spec, st)                   \
-                          : launch_d<DD, 4>(L, packed, x, y, grid, warps, rows_cap, smem, spec, st);
+        return units == 1 ? launch_d<DD, 1>(L, packed, x, y, grid, warps, rows_cap, smem, spec, gated ? 1 : 0, st)                   \
+             : units == 2 ? launch_d<DD, 2>(L, packed, x, y, grid, warps, rows_cap, smem, spec, gated ? 1 : 0, st)                   \
+                          : launch_d<DD, 4>(L, packed, x, y, grid, warps, rows_cap, smem, spec, gated ? 1 : 0, st);
     switch (depth) {
         PTQTP_LAUNCH_D(2)
         PTQTP_LAUNCH_D(3)

@@ -142,6 +142,8 @@ def config5(T):
                            ("down", 4096, 14336)]),
         ("stacked q/k/v and gate/up", [("qkv", 6144, 4096), ("o", 4096, 4096), ("gate_up", 28672, 4096),
                                        ("down", 4096, 14336)]),
+        ("stacked q/k/v, gate/up interleaved with the gated pair epilogue (ptqtp_gemv_swiglu)",
+         [("qkv", 6144, 4096), ("o", 4096, 4096), ("swiglu", 28672, 4096), ("down", 4096, 14336)]),
     ]
     for what, shapes in variants:
         base = {}
@@ -155,10 +157,14 @@ def config5(T):
         calls = []
         for l in range(copies):
             for name, N, K in shapes:
-                calls.append(lambda p=layers[l][name], N=N, K=K, x=base[name][1], y=base[name][2]:
-                             binding.ptqtp_gemv(p, N, K, x, y=y, stream=T.stream))
+                if name == "swiglu":
+                    calls.append(lambda p=layers[l][name], N=N, K=K, x=base[name][1], y=base[name][2][:N // 2]:
+                                 binding.ptqtp_gemv_swiglu(p, N, K, x, y=y, stream=T.stream))
+                else:
+                    calls.append(lambda p=layers[l][name], N=N, K=K, x=base[name][1], y=base[name][2]:
+                                 binding.ptqtp_gemv(p, N, K, x, y=y, stream=T.stream))
         us = T.steady_us(calls) * len(shapes)
-        nb = sum(algorithmic_bytes(N, K) for _, N, K in shapes)
+        nb = sum(algorithmic_bytes(N, K) - (N if name == "swiglu" else 0) for name, N, K in shapes)
         emit(workload="cfg5 llama3-8b layer, " + what, call="%d x ptqtp_gemv" % len(shapes), us_per_layer=round(us, 3),
              gbs=round(nb / us / 1e3, 1), bytes=nb, layer_copies=copies)
         del layers, base, calls

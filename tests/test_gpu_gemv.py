@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-from oracle.layer import layer_fp64
+from oracle.layer import layer_fp64, swiglu_fp64
 from paper_2509_16989_b200 import binding
 from paper_2509_16989_b200.inputs import (LLAMA3_70B, LLAMA3_8B_UNIQUE, QWEN3_0P6B_UP, make_activations,
                                           make_case, make_weights)
@@ -177,6 +177,42 @@ def test_stacked_matrices_give_the_rows_of_separate_calls():
     assert np.array_equal(ys[:1024].view(np.uint16), y1.view(np.uint16))
     assert np.array_equal(ys[1024:].view(np.uint16), y2.view(np.uint16))
     assert_parity(ys, oracle_y(stacked), stacked["x"], "stacked")
+
+
+@pytest.mark.parametrize("pairs,K", [(1, 128), (3, 1152), (64, 4096), (515, 2048), (1200, 4096), (300, 14336), (7168, 4096)])
+def test_gated_pair_epilogue_matches_oracle(pairs, K):
+    # rows 2i / 2i+1 = gate / up row i; y[i] = silu(gate) * up from the unrounded sums.  Error model: the two sums
+    # carry the GEMV's error B = 2e-3 * ||x||_inf * sqrt(K) at most (in practice about fp16 rounding of x's block
+    # fixed point), |silu'| <= 1.1, and the product is rounded once to fp16.
+    N = 2 * pairs
+    c = make_case(N, K, seed=900 + pairs)
+    c["alpha1"] = (c["alpha1"].astype(np.float32) * 4).astype(np.float16)          # gate values of order 1
+    packed = pack_case(c, binding.FORMAT_V2)
+    y = binding.ptqtp_gemv_swiglu(packed, N, K, dev(c["x"]))
+    torch.cuda.synchronize()
+    y = y.cpu().numpy().astype(np.float64)
+    t = layer_fp64(c["T1"], c["T2"], c["alpha1"], c["alpha2"], c["x"]) if pairs <= 600 else oracle_y(c)
+    g, u = t[0::2], t[1::2]
+    ref = g / (1.0 + np.exp(-g)) * u
+    if pairs <= 600:
+        assert np.allclose(ref, swiglu_fp64(c["T1"], c["T2"], c["alpha1"], c["alpha2"], c["x"]), rtol=1e-12, atol=1e-300)
+    B = 2e-3 * float(np.abs(c["x"].astype(np.float64)).max()) * np.sqrt(K)
+    bound = B * (1.1 * np.abs(u) + np.abs(g / (1.0 + np.exp(-g)))) + 2.0 ** -10 * np.abs(ref) + 1e-7
+    assert np.all(np.isfinite(y)) and y.shape == (pairs,)
+    assert np.all(np.abs(y - ref) <= bound)
+    assert np.linalg.norm(y - ref) <= 1e-3 * np.linalg.norm(ref) + 1e-6
+    # and it is exactly the epilogue applied to what ptqtp_gemv delivers before its fp16 rounding: compare with
+    # the epilogue applied to ptqtp_gemv's rounded outputs within fp16 resolution
+    yg = run_gemv(c, binding.FORMAT_V2).astype(np.float64)
+    approx = yg[0::2] / (1.0 + np.exp(-yg[0::2])) * yg[1::2]
+    assert np.all(np.abs(y - approx) <= 3 * 2.0 ** -10 * (np.abs(approx) + np.abs(yg[1::2]) * np.abs(yg[0::2]) * 1.1) + 1e-6)
+
+
+def test_gated_pair_epilogue_rejections():
+    c = make_case(5, 256, seed=1)
+    with pytest.raises(binding.PtqtpError) as e:
+        binding.ptqtp_gemv_swiglu(pack_case(c, binding.FORMAT_V2), 5, 256, dev(c["x"]))
+    assert e.value.status == binding.ERR_SHAPE
 
 
 def test_format2_rejects_format1_only_options():
