@@ -154,8 +154,9 @@ PTQTP_API ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape *shape /* host */, co
  * Format 2, M >= 2: the planes are contracted on the tensor cores with int8 warp MMAs against 15-bit
  * block-fixed-point activations (blocks of 128 columns), exact int32 sums, fp32 scale epilogue.  M = 2..4 take
  * one pass over the planes at about the cost of a batch-1 call (the activations stay in registers); larger M
- * decode the planes once per pass of up to 8 batch rows (fewer when K is long: the activations of a pass live
- * in shared memory).  M = 1 runs the batch-1 kernel.  Format 1: one batch-1 pass per row. */
+ * take one such pass per four rows (ptqtp_gemm_skinny_ws reads the planes once for any M).  When M rows of x
+ * leave no room in shared memory (very long K) a kernel that decodes the planes once per pass of up to 8 batch
+ * rows takes over.  M = 1 runs the batch-1 kernel.  Format 1: one batch-1 pass per row. */
 PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, const void *packed,
                                size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                void *stream);

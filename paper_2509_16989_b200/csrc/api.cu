@@ -150,12 +150,25 @@ ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, siz
     if (!aligned16(X) || !aligned16(Y)) return PTQTP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (L.v2) {
-        // two to four rows cost the same as one on the register-stationary tensor-core kernel
-        if (m >= 2 && m <= 4) {
-            const ptqtp_status s4 = launch_gemv3(L.l2, packed, m, X, Y, 0, 0, 0, st);
-            if (s4 != PTQTP_ERR_SHAPE) return s4;
+        // Up to four rows cost about the same as one on the register-stationary tensor-core kernel; more rows take
+        // one pass per four (ptqtp_gemm_skinny_ws reads the planes only once).  When four rows of x leave no room in
+        // shared memory the passes take three, two or, on the batch-1 kernel, one row.
+        if (m >= 2) {
+            int per_pass = m < 4 ? m : 4;
+            int done = 0;
+            while (done < m) {
+                const uint16_t* Xp = X + (size_t)done * shape->k_in;
+                uint16_t* Yp = Y + (size_t)done * shape->n_out;
+                const int rows = m - done < per_pass ? m - done : per_pass;
+                ptqtp_status sp = rows == 1 ? launch_gemv2(L.l2, packed, Xp, Yp, 0, 0, 0, 0, st)
+                                            : launch_gemv3(L.l2, packed, rows, Xp, Yp, 0, 0, 0, st);
+                if (sp == PTQTP_ERR_SHAPE && rows > 1 && done == 0) { --per_pass; continue; }   // nothing launched yet
+                if (sp != PTQTP_OK) return sp;
+                done += rows;
+            }
+            return PTQTP_OK;
         }
-        return m == 1 ? launch_gemv2(L.l2, packed, X, Y, 0, 0, 0, 0, st) : launch_skinny2(L.l2, packed, m, X, Y, st);
+        return launch_gemv2(L.l2, packed, X, Y, 0, 0, 0, 0, st);
     }
     return launch_gemm_skinny(L.l1, packed, m, X, Y, st);
 }

@@ -105,8 +105,6 @@ ptqtp_status launch_unpack2(const Layout2& L, const void* packed, int8_t* T1, in
                             uint16_t* a2, int32_t* dev_status, cudaStream_t st);
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
                           int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated = false);
-ptqtp_status launch_skinny2(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y,
-                            cudaStream_t st);
 size_t skinny3_workspace_bytes(int k, int m);
 ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, void* workspace,
                             cudaStream_t st);

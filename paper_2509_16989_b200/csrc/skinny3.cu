@@ -1,16 +1,16 @@
 // Small-batch dual-trit-plane GEMM with a caller-provided workspace (format 2):  Y[m,:] = layer(X[m,:]), M <= 64.
 //
-// Same contraction as skinny2.cu (int8 warp MMAs on masked codes x block-fixed-point activations), organised so
+// Same contraction as gemv3.cu (int8 warp MMAs on masked codes x block-fixed-point activations), organised so
 // that the packed planes are read from HBM exactly once for any M and any K:
 //
 //   * A first kernel converts X once into the workspace: for every 1024-column half slice the rows
 //     (2j = high byte, 2j + 1 = low byte of batch row j) as 1024 contiguous bytes each, and one record
-//     (2^-s, sum of the block's integers) per batch row and 128-column block.  In skinny2.cu every CTA repeats
-//     this conversion and keeps the result for all K in shared memory, which caps a pass at 1 to 8 batch rows.
+//     (2^-s, sum of the block's integers) per batch row and 128-column block.  (In gemv3.cu every CTA repeats
+//     this conversion for its one to four rows.)
 //   * The main kernel gives each warp one quad of four row pairs per round and walks the half slices in order,
 //     the whole CTA in step: the activation tile of a step (one half slice, up to 16 batch rows) is copied from
 //     the workspace (L2-resident) into shared memory by all threads, double buffered, while the warps' code
-//     units stream through per-warp ring slots as before.  A warp keeps the row sums of its quad for all
+//     units stream through per-warp ring slots.  A warp keeps the row sums of its quad for all
 //     batch rows in registers across the half slices, so no partial sums go through shared memory and the
 //     result is written once at the end of the round.
 //   * The main kernel issues its first code copies before griddepcontrol.wait, i.e. while the conversion kernel
