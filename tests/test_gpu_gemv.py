@@ -505,6 +505,29 @@ def test_overlapped_chain_keeps_stream_order(graph, level):
         binding.ptqtp_set_overlap(2)
 
 
+@pytest.mark.parametrize("level", [0, 1])
+def test_other_overlap_levels_on_ragged_and_long_shapes(level):
+    # level 0: plain launches with whole-SM CTAs; level 1: dependent launch without speculative execution
+    old = binding.ptqtp_set_overlap(level)
+    try:
+        for N, K in ((5, 1152), (1000, 14336), (37, 36864), (4097, 6144), (2, 128)):
+            c = make_case(N, K, seed=300 + N, M=3)
+            packed = pack_case(c, binding.FORMAT_V2)
+            y = binding.ptqtp_gemv(packed, N, K, dev(c["x"][0].copy()), fmt=binding.FORMAT_V2)
+            Y = binding.ptqtp_gemm_skinny(packed, N, K, dev(c["x"]), fmt=binding.FORMAT_V2)
+            g = binding.ptqtp_gemv_swiglu(packed, N, K, dev(c["x"][1].copy())) if N % 2 == 0 else None
+            torch.cuda.synchronize()
+            ref = oracle_y(c)
+            assert_parity(y.cpu().numpy(), ref[0], c["x"][0], "level %d gemv N=%d K=%d" % (level, N, K))
+            assert_parity(Y.cpu().numpy(), ref, c["x"], "level %d skinny N=%d K=%d" % (level, N, K))
+            if g is not None:
+                t = ref[1]
+                want = t[0::2] / (1.0 + np.exp(-t[0::2])) * t[1::2]
+                assert np.linalg.norm(g.cpu().numpy().astype(np.float64) - want) <= 1e-3 * np.linalg.norm(want) + 1e-6
+    finally:
+        binding.ptqtp_set_overlap(old)
+
+
 def test_speculative_read_sees_activations_written_just_before():
     # x is rewritten on the stream (by a copy, by an elementwise kernel) directly before each call, alternating
     # between two vectors that differ in one element only; every call must use the value written last.
