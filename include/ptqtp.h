@@ -196,8 +196,11 @@ PTQTP_API ptqtp_status ptqtp_gemm_skinny_static(const ptqtp_shape *shape /* host
                                       void *stream);
 
 /* End-to-end convenience for callers holding activations on the host: copies x_host [K] (host,
- * ideally pinned) to x_dev, runs ptqtp_gemv, copies y_dev to y_host [N]; all three enqueued on
- * `stream`, no synchronisation.  x_dev [K] and y_dev [N] are caller-owned device staging buffers. */
+ * ideally pinned) to x_dev, runs ptqtp_gemv and delivers y in y_host [N]; everything is enqueued on
+ * `stream`, no synchronisation: y_host is valid once the stream has reached this point.  x_dev [K] and
+ * y_dev [N] are caller-owned device staging buffers.  When y_host is pinned, 16-byte aligned memory that the
+ * device can address (format 2), the kernel stores y there directly and y_dev is left untouched; otherwise
+ * y is computed into y_dev and copied to y_host. */
 PTQTP_API ptqtp_status ptqtp_gemv_host(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                              const uint16_t *x_host, uint16_t *y_host, uint16_t *x_dev, uint16_t *y_dev,
                              void *stream);

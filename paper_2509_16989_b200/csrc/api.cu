@@ -219,11 +219,28 @@ ptqtp_status ptqtp_gemv_host(const ptqtp_shape* shape, const void* packed, size_
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)shape->k_in * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+    // When y_host is pinned memory that the device can address (any pinned allocation under unified addressing),
+    // the kernel stores y there itself and the copy back is saved; otherwise y goes through y_dev.
+    uint16_t* y_target = y_dev;
+    bool direct = false;
+    if (L.v2 && aligned16(y_host)) {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, y_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+            attr.devicePointer != nullptr) {
+            y_target = static_cast<uint16_t*>(attr.devicePointer);
+            direct = true;
+        } else {
+            (void)cudaGetLastError();                    // pageable memory: not an error for this call
+        }
+    }
     // between its two copies the kernel never overlaps another GEMV: it gets whole SMs
-    s = L.v2 ? launch_gemv2(L.l2, packed, x_dev, y_dev, -1, 0, 0, 0, st) : gemv_any(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
+    s = L.v2 ? launch_gemv2(L.l2, packed, x_dev, y_target, -1, 0, 0, 0, st)
+             : gemv_any(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
     if (s != PTQTP_OK) return s;
-    e = cudaMemcpyAsync(y_host, y_dev, (size_t)shape->n_out * 2, cudaMemcpyDeviceToHost, st);
-    if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+    if (!direct) {
+        e = cudaMemcpyAsync(y_host, y_dev, (size_t)shape->n_out * 2, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+    }
     return PTQTP_OK;
 }
 

@@ -426,10 +426,21 @@ def test_gemv_host_entry_point(fmt):
     y_host = torch.empty(300, dtype=torch.float16).pin_memory()
     x_dev = torch.empty(2048, dtype=torch.float16, device="cuda")
     y_dev = torch.empty(300, dtype=torch.float16, device="cuda")
+    y_dev.fill_(-7.0)
     binding.ptqtp_gemv_host(packed, 300, 2048, x_host, y_host, x_dev, y_dev, fmt=fmt)
     torch.cuda.synchronize()
     assert_parity(y_host.numpy(), oracle_y(c), c["x"], "host call")
-    assert np.array_equal(y_host.numpy().view(np.uint16), y_dev.cpu().numpy().view(np.uint16))
+    if fmt == binding.FORMAT_V2:
+        # pinned y_host: the kernel stores y there itself and leaves the staging buffer alone
+        assert bool((y_dev == -7.0).all())
+    else:
+        assert np.array_equal(y_host.numpy().view(np.uint16), y_dev.cpu().numpy().view(np.uint16))
+    # pageable y_host: through the staging buffer, same bits
+    y_page = torch.empty(300, dtype=torch.float16)
+    binding.ptqtp_gemv_host(packed, 300, 2048, x_host, y_page, x_dev, y_dev, fmt=fmt)
+    torch.cuda.synchronize()
+    assert np.array_equal(y_page.numpy().view(np.uint16), y_host.numpy().view(np.uint16))
+    assert np.array_equal(y_page.numpy().view(np.uint16), y_dev.cpu().numpy().view(np.uint16))
 
 
 def test_decomposed_weights_end_to_end():
