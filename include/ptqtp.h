@@ -244,11 +244,12 @@ PTQTP_API ptqtp_status ptqtp_kernel_status(int32_t *status_host /* host */, void
 
 /* Overlap of consecutive GEMV calls on one stream (process-wide level, default 2; returns the old level).
  * Level 0: plain launches.  Level 1: format-2 GEMV kernels are launched with programmatic stream
- * serialization: a call may begin reading its `packed` blob while the GEMV call directly before it on the
+ * serialization: a call may begin reading its `packed` blob while the kernel directly before it on the
  * stream is still draining; x is used and y written only after all earlier work on the stream has completed,
- * so stream order holds for them.  Consequence for the caller: the packed blob of a call must not be the
- * output buffer of the GEMV call directly before it.  Work of any other kind before a call is always complete
- * before the call reads anything.  Works inside CUDA graph capture.
+ * so stream order holds for them.  Consequence for the caller: the packed blob of a call must be complete
+ * before the kernel directly ahead of the call on its stream ends -- it must not be the output buffer of that
+ * kernel.  ptqtp_pack is exempt (the first GEMV call after a ptqtp_pack on the same stream is a plain launch),
+ * and so are copies (cudaMemcpyAsync and the like are not kernels).  Works inside CUDA graph capture.
  * Level 2 adds speculative execution: the kernel reads x at once and computes everything into shared memory
  * while earlier work of the stream may still be running, then waits for that work, reads x again and compares
  * it bit by bit with its first read; y is written only after that, and if a single bit of x differed the whole

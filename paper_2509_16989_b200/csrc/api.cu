@@ -1,5 +1,7 @@
 // C ABI of libptqtp: argument validation and dispatch.  Declarations and contracts: include/ptqtp.h.
 #include <string.h>
+#include <mutex>
+#include <vector>
 #include "ptqtp_internal.h"
 
 namespace ptqtp {
@@ -8,6 +10,33 @@ static thread_local int g_last_cuda_error = 0;
 static int g_overlap = 2;
 
 bool overlap_enabled() { return g_overlap != 0; }
+
+// Streams on which ptqtp_pack was the library's last call: the next GEMV launch there is a plain launch, so that
+// it reads the packed planes only after the pack kernel has completed (a dependent launch reads them earlier).
+static std::mutex g_pack_mutex;
+static std::vector<cudaStream_t> g_pack_streams;
+static bool g_pack_overflow = false;
+void note_pack(cudaStream_t st) {
+    std::lock_guard<std::mutex> lock(g_pack_mutex);
+    for (cudaStream_t s : g_pack_streams)
+        if (s == st) return;
+    if (g_pack_streams.size() < 256) g_pack_streams.push_back(st); else g_pack_overflow = true;
+}
+bool consume_pack(cudaStream_t st) {
+    std::lock_guard<std::mutex> lock(g_pack_mutex);
+    if (g_pack_overflow) {                              // too many streams to remember: be plain once everywhere
+        g_pack_overflow = false;
+        g_pack_streams.clear();
+        return true;
+    }
+    for (size_t i = 0; i < g_pack_streams.size(); ++i) {
+        if (g_pack_streams[i] == st) {
+            g_pack_streams.erase(g_pack_streams.begin() + i);
+            return true;
+        }
+    }
+    return false;
+}
 bool speculation_enabled() { return g_overlap >= 2; }
 
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
@@ -93,6 +122,7 @@ ptqtp_status ptqtp_pack(const ptqtp_shape* shape, const int8_t* T1, const int8_t
     if (!aligned16(T1) || !aligned16(T2) || !aligned16(alpha1) || !aligned16(alpha2)) return PTQTP_ERR_ALIGN;
     if (dev_status && (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return PTQTP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    note_pack(st);
     return L.v2 ? launch_pack2(L.l2, T1, T2, alpha1, alpha2, packed, dev_status, st)
                 : launch_pack(L.l1, T1, T2, alpha1, alpha2, packed, dev_status, st);
 }

@@ -429,7 +429,7 @@ ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, u
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = overlap_enabled() ? 1 : 0;
+    cfg.numAttrs = overlap_enabled() && !consume_pack(st) ? 1 : 0;   // plain right after a pack on this stream
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, L, static_cast<const unsigned char*>(packed),
                                        reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap,
                                        L.nrp / grid, L.nrp % grid, speculate, gated);

@@ -472,7 +472,7 @@ ptqtp_status launch_gemv3(const Layout2& L, const void* packed, int m, const uin
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = overlap_enabled() ? 1 : 0;
+    cfg.numAttrs = overlap_enabled() && !consume_pack(st) ? 1 : 0;   // plain right after a pack on this stream
     cudaError_t e = cudaLaunchKernelEx(&cfg, gemv3_kernel, L, static_cast<const unsigned char*>(packed),
                                        reinterpret_cast<const __half*>(X), reinterpret_cast<__half*>(Y), m, rows_cap,
                                        nquads / grid, nquads % grid, teams, depth, speculate, status_word);

@@ -117,5 +117,6 @@ ptqtp_status launch_gemv3(const Layout2& L, const void* packed, int m, const uin
 int sm_count();
 bool speculation_enabled();       // speculative read of x before the dependency wait (ptqtp_set_overlap(2))
 bool overlap_enabled();           // programmatic dependent launch of the GEMV kernels (ptqtp_set_overlap)
+bool consume_pack(cudaStream_t st);   // true once after ptqtp_pack on this stream: the next GEMV launch is plain
 
 }  // namespace ptqtp

@@ -539,6 +539,28 @@ def test_other_overlap_levels_on_ragged_and_long_shapes(level):
         binding.ptqtp_set_overlap(old)
 
 
+def test_pack_directly_before_a_call_on_the_same_stream():
+    # the same packed buffer is rewritten by ptqtp_pack and used by the next call without any synchronisation
+    N, K = 2048, 4096
+    cs = [make_case(N, K, seed=80 + i) for i in range(2)]
+    for c in cs:
+        c["x"] = cs[0]["x"]
+    planes = [tuple(dev(c[k]) for k in ("T1", "T2", "alpha1", "alpha2")) for c in cs]
+    packed = torch.empty(binding.packed_size(N, K), dtype=torch.uint8, device="cuda")
+    x = dev(cs[0]["x"])
+    ys = [torch.empty(N, dtype=torch.float16, device="cuda") for _ in range(8)]
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for i, y in enumerate(ys):
+            binding.ptqtp_pack(*planes[i % 2], packed=packed, stream=stream)
+            binding.ptqtp_gemv(packed, N, K, x, y=y, stream=stream)
+        stream.synchronize()
+    refs = [oracle_y(c) for c in cs]
+    for i, y in enumerate(ys):
+        assert_parity(y.cpu().numpy(), refs[i % 2], cs[0]["x"], "call %d" % i)
+    assert not np.array_equal(ys[0].cpu().numpy().view(np.uint16), ys[1].cpu().numpy().view(np.uint16))
+
+
 def test_speculative_read_sees_activations_written_just_before():
     # x is rewritten on the stream (by a copy, by an elementwise kernel) directly before each call, alternating
     # between two vectors that differ in one element only; every call must use the value written last.
