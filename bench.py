@@ -36,7 +36,7 @@ UNIQUE_OF = {"q": "qo", "o": "qo", "k": "kv", "v": "kv", "gate": "gate_up", "up"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes in the ncu capture of the 14336x4096 launch of
 # the current GEMV kernel (profiles/gemv2_gate_up_14336x4096.md); set to None when the kernel changes
-DRAM_TRAFFIC_RATIO = 31232000.0 / 31232000.0
+DRAM_TRAFFIC_RATIO = 31239424.0 / 31232000.0
 FALLBACK_HBM_GBS = 6650.0
 
 

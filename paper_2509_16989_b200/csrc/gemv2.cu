@@ -314,15 +314,14 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                 }
                 const int nun = min(RU, n_rp - j0);
                 const unsigned char* buf = ring + cslot * kSlot + ln * 16;
-#pragma unroll 1
-                for (int u = 0; u < nun; ++u, buf += ubytes) {
+                auto unit_body = [&](const unsigned char* ub, float* pp) {
                 // Fields 0..2 are masked out of each code word; the unmasked word gives the sum of all four fields
                 // (a byte is q0 + 4 q1 + 16 q2 + 64 q3 <= 170), so field 3 is "all" minus the other three.
                 int ah[4] = {0, 0, 0, 0};
                 int al[4] = {n0, n1, n2, n3};
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const uint4 cw = *reinterpret_cast<const uint4*>(buf + i * atom_stride);
+                    const uint4 cw = *reinterpret_cast<const uint4*>(ub + i * atom_stride);
                     const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
                     for (int ww = 0; ww < 4; ++ww) {
@@ -336,7 +335,7 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                         al[3] = dot_uu(w[ww], xl[4 * i + ww], al[3]);
                     }
                 }
-                const uint2 sc = *reinterpret_cast<const uint2*>(buf + scale_off);
+                const uint2 sc = *reinterpret_cast<const uint2*>(ub + scale_off);
                 const float2 s0 = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));   // alpha1, alpha2 of row 0
                 const float2 s1 = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));   // ... of row 1
                 // Q0..Q2 = 4^f * sum_j t_j X_j of fields 0..2; the unmasked word minus those three is field 3's
@@ -351,8 +350,17 @@ gemv2_kernel(Layout2 L, const unsigned char* __restrict__ packed, const __half* 
                 float v = ((lane & 16) ? y1 : y0) + __shfl_xor_sync(0xffffffffu, send, 16);
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if ((lane & 15) == 0) *ppart = failed ? __int_as_float(0x7fc00000) : v;
-                ppart += 2 * S;
+                if ((lane & 15) == 0) *pp = failed ? __int_as_float(0x7fc00000) : v;
+                };
+                if (RU == 2 && nun == 2) {
+                    // both units in one basic block: the second unit's loads and dot products fill the latencies of
+                    // the first unit's epilogue and reduction
+                    unit_body(buf, ppart);
+                    unit_body(buf + ubytes, ppart + 2 * S);
+                    ppart += 4 * S;
+                } else {
+#pragma unroll 1
+                    for (int u = 0; u < nun; ++u, buf += ubytes, ppart += 2 * S) unit_body(buf, ppart);
                 }
                 // every lane has consumed the slot: lane 0 may refill it
                 __syncwarp();
