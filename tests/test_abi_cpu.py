@@ -97,6 +97,14 @@ def test_host_side_validation_codes(L):
     assert L.ptqtp_pack(sp, ok_ptr, odd_ptr, ok_ptr, ok_ptr, ok_ptr, size, None, None) == binding.ERR_ALIGN
     assert L.ptqtp_unpack(sp, ok_ptr, size - 4, ok_ptr, ok_ptr, ok_ptr, ok_ptr, None, None) == binding.ERR_SIZE
     assert L.ptqtp_gemv_host(sp, ok_ptr, size, None, ok_ptr, ok_ptr, ok_ptr, None) == binding.ERR_NULL
+    # gated pair epilogue: format 2 only, an even number of rows
+    assert L.ptqtp_gemv_swiglu(sp, ok_ptr, size, None, ok_ptr, None) == binding.ERR_NULL
+    assert L.ptqtp_gemv_swiglu(sp, ok_ptr, size, ok_ptr, odd_ptr, None) == binding.ERR_ALIGN
+    odd_rows = binding.make_shape(7, 256)
+    assert L.ptqtp_gemv_swiglu(ctypes.byref(odd_rows), ok_ptr, size, ok_ptr, ok_ptr, None) == binding.ERR_SHAPE
+    v1 = binding.make_shape(8, 256, fmt=binding.FORMAT_V1)
+    assert L.ptqtp_gemv_swiglu(ctypes.byref(v1), ok_ptr, binding.packed_size(8, 256, fmt=binding.FORMAT_V1), ok_ptr, ok_ptr,
+                               None) == binding.ERR_CONFIG
 
 
 def test_status_strings(L):
