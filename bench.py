@@ -117,20 +117,26 @@ class ClockSampler(threading.Thread):
         except Exception:
             self._h = None
 
-    def run(self):
+    def sample_now(self):
+        """One sample taken by the caller (a short timed region may end before the thread's next turn)."""
         if self._h is None:
             return
         nv = self._nv
-        while not self._stop_evt.is_set():
+        try:
+            mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
             try:
-                mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
-                try:
-                    rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
-                except Exception:
-                    rs = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
-                self.samples.append((time.perf_counter(), mhz, rs))
+                rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
             except Exception:
-                pass
+                rs = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+            self.samples.append((time.perf_counter(), mhz, rs))
+        except Exception:
+            pass
+
+    def run(self):
+        if self._h is None:
+            return
+        while not self._stop_evt.is_set():
+            self.sample_now()
             self._stop_evt.wait(0.02)
 
     def stop(self):
@@ -139,7 +145,7 @@ class ClockSampler(threading.Thread):
     def summary(self, t0, t1):
         inside = [s for s in self.samples if t0 <= s[0] <= t1]
         window = "timed region"
-        if len(inside) < 3:
+        if len(inside) < 3 and len(self.samples) > len(inside):
             inside = list(self.samples)
             window = "whole run (timed region shorter than 3 samples)"
         if not inside:
@@ -272,6 +278,7 @@ def run_gpu(args):
     stream.synchronize()
     graphs = None
     big = None
+    huge = None
     if not args.no_graph:
         graphs = []
         for r in range(R):
@@ -283,6 +290,17 @@ def run_gpu(args):
         with torch.cuda.graph(big, stream=stream):
             for r in range(R):
                 step(r)
+        # eight rotations in one graph: a graph boundary drains the chain of overlapping launches
+        huge = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(huge, stream=stream):
+            for _ in range(8):
+                for r in range(R):
+                    step(r)
+        # first replays upload the graphs to the device: part of the set-up, like packing the matrices
+        with torch.cuda.stream(stream):
+            for g in graphs + [big, huge]:
+                g.replay()
+        stream.synchronize()
 
     def run_steps(k, start=0):
         with torch.cuda.stream(stream):
@@ -295,6 +313,9 @@ def run_gpu(args):
             while i < k and (start + i) % R != 0:
                 graphs[(start + i) % R].replay()
                 i += 1
+            while k - i >= 8 * R:
+                huge.replay()
+                i += 8 * R
             while k - i >= R:
                 big.replay()
                 i += R
@@ -319,6 +340,7 @@ def run_gpu(args):
     e0.record(stream)
     run_steps(args.steps)
     e1.record(stream)
+    sampler.sample_now()                                 # the GPU is still working on the enqueued steps
     stream.synchronize()
     torch.cuda.synchronize()
     t_end = time.perf_counter()
