@@ -8,6 +8,7 @@
   5  a LLaMA-3-8B layer with stacked matrices: q, k, v packed as one 6144 x 4096 matrix, and also gate, up as one
      28672 x 4096 matrix (rows are independent, so a caller may stack matrices that share their input and
      slice y): five or four calls per layer instead of seven
+  6  the seven linears of a LLaMA-3-70B-shaped layer as one chain of calls
 
 (The 32-layer stack built from decomposed weights needs the CPU oracle to prepare its inputs and is therefore
 measured by tests/test_gpu_stack.py.)
@@ -171,9 +172,30 @@ def config5(T):
         torch.cuda.empty_cache()
 
 
+def config6(T):
+    # the seven linears of a LLaMA-3-70B-shaped layer as one chain of calls, two copies of the layer (> 2x L2)
+    order = [("q", "qo"), ("k", "kv"), ("v", "kv"), ("o", "qo"), ("gate", "gate_up"), ("up", "gate_up"), ("down", "down")]
+    base = {}
+    for i, u in enumerate(sorted(LLAMA3_70B)):
+        N, K = LLAMA3_70B[u]
+        c = make_case(N, K, seed=60 + i)
+        packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
+        base[u] = (packed, dev(c["x"]), torch.empty(N, dtype=torch.float16, device="cuda"))
+    calls = []
+    for l in range(2):
+        for name, u in order:
+            p = base[u][0] if (l == 0 and name in ("q", "k", "gate", "down")) else base[u][0].clone()
+            N, K = LLAMA3_70B[u]
+            calls.append(lambda p=p, N=N, K=K, x=base[u][1], y=base[u][2]: binding.ptqtp_gemv(p, N, K, x, y=y, stream=T.stream))
+    us = T.steady_us(calls, reps=40) * len(order)
+    nb = sum(algorithmic_bytes(*LLAMA3_70B[u]) for _, u in order)
+    emit(workload="cfg6 llama3-70b-shaped layer as one chain", call="7 x ptqtp_gemv", us_per_layer=round(us, 3),
+         gbs=round(nb / us / 1e3, 1), bytes=nb, layer_copies=2)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="0,2,3,5")
+    ap.add_argument("--only", default="0,2,3,5,6")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise RuntimeError("needs a CUDA device")
@@ -188,6 +210,8 @@ def main():
         config3(T)
     if 5 in which:
         config5(T)
+    if 6 in which:
+        config6(T)
 
 
 if __name__ == "__main__":
