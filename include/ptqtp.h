@@ -63,6 +63,24 @@
  *                       A full slice unit is 2048 + 128 = 2176 bytes.
  *   ptqtp_packed_size = 256 + ceil(N/2) * (K + K/16 rounded up per unit) bytes; for even N and K % 256 == 0
  *   exactly the Appendix B figure plus the header.
+ *
+ * Packed format 3 (same storage model; the code bytes of format 2 laid out in the operand order of the int8
+ * warp-level matrix instruction, so that the batch-1 kernel decodes with three masks per code word):
+ *   [0, 256)            header as above with format(3); the K_pad slot holds 512 * ceil(K/512) and the
+ *                       scales_offset slot holds the bytes of one tile (4352).
+ *   body  (at 256)      tiles of 8 row pairs (16 rows) x 512 columns (four 128-column groups), 4352 bytes each,
+ *                       superblock-major: tile (sb, rb) -- columns 512 sb .., row pairs 8 rb .. -- at byte
+ *                       256 + (sb * ceil(ceil(N/2)/8) + rb) * 4352, so the tiles of one 512-column superblock for
+ *                       consecutive row blocks are contiguous.  Rows >= N and columns >= K are stored as trit 0
+ *                       with scales 0.  A tile:
+ *                         codes   8 chunks of 512 bytes; chunk c holds for lane l = 4 g + t (g = 0..7 the row pair
+ *                                 within the tile, t = 0..3) 16 bytes at 512 c + 16 l = four words (s, h) at byte
+ *                                 8 s + 4 h; byte e of word (s, h) is the column byte (as in format 2) of row pair
+ *                                 8 rb + g and column 512 sb + 128 (2 h + t / 2) + 8 (2 c + s) + 4 (t % 2) + e.
+ *                         scales  32 quads of 8 bytes at byte 4096 + 8 l: fp16 alpha1[2p], alpha2[2p], alpha1[2p+1],
+ *                                 alpha2[2p+1] of row pair p = 8 rb + g and group 4 sb + t.
+ *   ptqtp_packed_size = 256 + ceil(ceil(N/2)/8) * ceil(K/512) * 4352 bytes; for N % 16 == 0 and K % 512 == 0
+ *   exactly the Appendix B figure plus the header.
  */
 #ifndef PTQTP_H
 #define PTQTP_H
@@ -96,12 +114,13 @@ typedef struct {
     int32_t n_out;   /* N: output features (rows of W)            */
     int32_t k_in;    /* K: input features, multiple of 128        */
     int32_t group;   /* scale group size along K; must be 128     */
-    int32_t format;  /* packed format id: 1 or 2                  */
+    int32_t format;  /* packed format id: 1, 2 or 3               */
 } ptqtp_shape;
 
 #define PTQTP_GROUP 128
 #define PTQTP_FORMAT_V1 1
 #define PTQTP_FORMAT_V2 2
+#define PTQTP_FORMAT_V3 3
 #define PTQTP_HEADER_BYTES 256
 #define PTQTP_MAX_BATCH 64
 #define PTQTP_STATIC_WORKSPACE_BYTES (512 * 1024)
@@ -134,8 +153,10 @@ PTQTP_API ptqtp_status ptqtp_unpack(const ptqtp_shape *shape /* host */, const v
  * Arithmetic, format 1: fp16 x times codes, fp32 accumulators, fp32 scale epilogue.
  * Arithmetic, format 2: x is turned into 16-bit block fixed point per 64 columns (exact for values within
  * 2^-5 of the block maximum, otherwise rounded to 2^-16 of it), sign-select sums are exact int32, the
- * scale epilogue and the sums over groups are fp32.  One rounding to fp16 at the store in both.
- * Non-finite x gives unspecified y. */
+ * scale epilogue and the sums over groups are fp32.  Arithmetic, format 3: x is turned into 15-bit block fixed
+ * point per 128-column group (rounded to 2^-14 of the group maximum), the sign-select sums are contracted by
+ * int8 warp-level matrix instructions and are exact int32, the scale epilogue and the sums over groups are fp32.
+ * One rounding to fp16 at the store in all three.  Non-finite x gives unspecified y. */
 PTQTP_API ptqtp_status ptqtp_gemv(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                         const uint16_t *x, uint16_t *y, void *stream);
 
@@ -144,7 +165,7 @@ PTQTP_API ptqtp_status ptqtp_gemv(const ptqtp_shape *shape /* host */, const voi
  * ONE matrix of N rows (N even) that holds the gate and up projections interleaved by rows: row 2i = gate row i,
  * row 2i+1 = up row i.  With t = the layer's N fp32 row sums (before any rounding to fp16),
  *     y[i] = silu(t[2i]) * t[2i+1],   silu(g) = g / (1 + exp(-g)),   i < N/2,
- * rounded once to fp16.  y: device fp16 [N/2].  Format 2 only (PTQTP_ERR_CONFIG for format 1); PTQTP_ERR_SHAPE for
+ * rounded once to fp16.  y: device fp16 [N/2].  Formats 2 and 3 (PTQTP_ERR_CONFIG for format 1); PTQTP_ERR_SHAPE for
  * odd N.  Everything else as ptqtp_gemv (same kernel: only its final store differs). */
 PTQTP_API ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                                const uint16_t *x, uint16_t *y, void *stream);
@@ -154,9 +175,10 @@ PTQTP_API ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape *shape /* host */, co
  * Format 2, M >= 2: the planes are contracted on the tensor cores with int8 warp MMAs against 15-bit
  * block-fixed-point activations (blocks of 128 columns), exact int32 sums, fp32 scale epilogue.  M = 2..4 take
  * one pass over the planes at about the cost of a batch-1 call (the activations stay in registers); larger M
- * take one such pass per four rows (ptqtp_gemm_skinny_ws reads the planes once for any M).  When M rows of x
- * leave no room in shared memory (very long K) a kernel that decodes the planes once per pass of up to 8 batch
- * rows takes over.  M = 1 runs the batch-1 kernel.  Format 1: one batch-1 pass per row. */
+ * take one such pass per four rows (ptqtp_gemm_skinny_ws reads the planes once for any M).  When four rows of x
+ * leave no room in shared memory (very long K) the passes take three or two rows, or one row on the batch-1
+ * kernel.  M = 1 runs the batch-1 kernel.  Formats 1 and 3 are batch-1 layouts: M = 1 runs their batch-1 kernel,
+ * M > 1 returns PTQTP_ERR_CONFIG (pack a format-2 blob for small batches). */
 PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, const void *packed,
                                size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                void *stream);
@@ -167,7 +189,7 @@ PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, co
  * converted once to block fixed point; with it the packed planes are read from HBM exactly once for any M and
  * K, where ptqtp_gemm_skinny needs several passes when M or K is large.  Two kernels are enqueued on `stream`.
  * Calls that share a workspace must not overlap on the GPU.  ptqtp_gemm_skinny_workspace_size returns 0 for a
- * bad shape, format 1 or M out of range.  Batch sweep of the benchmark spec's small-batch call list. */
+ * bad shape, formats 1 and 3 or M out of range.  (Small-batch use of the layer of Eq. 1-2; the paper measures batch 1.) */
 PTQTP_API size_t ptqtp_gemm_skinny_workspace_size(const ptqtp_shape *shape /* host */, int32_t m);
 PTQTP_API ptqtp_status ptqtp_gemm_skinny_ws(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                                   int32_t m, const uint16_t *X, uint16_t *Y, void *workspace,
@@ -220,7 +242,11 @@ PTQTP_API ptqtp_status ptqtp_gemv_host(const ptqtp_shape *shape /* host */, cons
  * together; 16 serves a call that runs alone best); ctas_per_sm = CTAs of this launch per SM (1..4, 0 = 1);
  * depth = copies in flight per warp (2, 3, 4, 6, 8; 0 = 2).  arith 4: rows_per_warp must be 0; k_split = warps
  * per CTA (4, 8 or 16, 0 = auto); ctas_per_sm 1 or 2 (0 = 1); depth = stages (four slice units each) per team of
- * four warps (2..8, 0 = auto).  A configuration that does not fit in shared memory gives PTQTP_ERR_CONFIG. */
+ * four warps (2..8, 0 = auto).  A configuration that does not fit in shared memory gives PTQTP_ERR_CONFIG.
+ * For a format-3 blob: arith = -1 or 5; rows_per_warp = tiles per bulk copy (1 or 2, 0 = library choice);
+ * k_split = warps per CTA (1..16 / ctas_per_sm, 0 = library choice, -1 = as many as have work: for a call that runs
+ * alone); ctas_per_sm = CTAs of this launch per SM (1..4, 0 = 1); depth = copies in flight per warp (2, 3, 4, 6;
+ * 0 = library choice). */
 PTQTP_API ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                             const uint16_t *x, uint16_t *y, int32_t rows_per_warp, int32_t k_split,
                             int32_t ctas_per_sm, int32_t depth, int32_t arith, void *stream);
@@ -235,15 +261,31 @@ PTQTP_API const char *ptqtp_status_string(ptqtp_status status);
 /* The cudaError_t (as int) behind the calling thread's most recent PTQTP_ERR_CUDA, else 0. */
 PTQTP_API int ptqtp_last_cuda_error(void);
 
-/* Device-side health of the format-2 kernels that stream the packed planes with bulk copies (batch 1, and the
- * small-batch kernel for two to four rows) on the current device.  They wait for each copy with a bounded
+/* Device-side health of the kernels that stream the packed planes with bulk copies (batch 1 of formats 2 and 3,
+ * and the small-batch kernel for two to four rows) on the current device.  They wait for each copy with a bounded
  * number of polls; if a wait ever gives up, the kernel
  * writes NaN to the rows it could not finish, records PTQTP_ERR_CUDA in a device word and still terminates.
  * This call enqueues a copy of that word (0 = healthy) to *status_host on `stream`; read it after syncing. */
 PTQTP_API ptqtp_status ptqtp_kernel_status(int32_t *status_host /* host */, void *stream);
 
-/* Overlap of consecutive GEMV calls on one stream (process-wide level, default 2; returns the old level).
- * Level 0: plain launches.  Level 1: format-2 GEMV kernels are launched with programmatic stream
+/* Reset that device word to 0 (enqueued on `stream`): the word is only ever set by the kernels, so after a
+ * reported failure it keeps its value until this call. */
+PTQTP_API ptqtp_status ptqtp_kernel_status_clear(void *stream);
+
+/* Number of polls after which a bounded wait for a bulk copy gives up (process-wide, default 2^22, at least 1;
+ * returns the old value).  A poll takes from tens of nanoseconds to a few microseconds. */
+PTQTP_API int ptqtp_set_wait_limit(int polls);
+
+/* Test hook for the give-up path of the bounded waits: each of the next `launches` format-3 batch-1 launches
+ * announces, on one mbarrier of its first CTA, 16 bytes more than the copy brings, so that wait runs out after
+ * ptqtp_set_wait_limit polls: the affected rows come out as NaN and ptqtp_kernel_status reports PTQTP_ERR_CUDA.
+ * Every copy still lands and the kernel ends normally.  Not for production use. */
+PTQTP_API void ptqtp_test_fail_next_wait(int launches);
+
+/* Overlap of consecutive GEMV calls on one stream (process-wide level, default 0; returns the old level).
+ * Level 0 (default): plain launches; every buffer, `packed` included, follows stream order.  Levels 1 and 2 are
+ * an opt-in for callers whose packed blobs are immutable while GEMV calls are in flight (the decode case).
+ * Level 1: the GEMV kernels of formats 2 and 3 are launched with programmatic stream
  * serialization: a call may begin reading its `packed` blob while the kernel directly before it on the
  * stream is still draining; x is used and y written only after all earlier work on the stream has completed,
  * so stream order holds for them.  Consequence for the caller: the packed blob of a call must be complete

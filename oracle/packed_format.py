@@ -24,6 +24,20 @@ bytes of one row pair over all slices):
                    alpha1[2p+1], alpha2[2p+1]) for the slice's 128-column groups; then zero padding to a
                    multiple of 16 bytes.
 
+Format 3 (same header with format = 3; the K_pad slot holds 512 * ceil(K/512), the scales-offset slot the bytes of
+one tile, 4352):
+
+  body             tiles of 8 row pairs (16 rows) x 512 columns (four 128-column groups), 4352 bytes each, stored
+                   superblock-major: tile (sb, rb) -- columns 512 sb .., row pairs 8 rb .. -- at byte
+                   256 + (sb * ceil(ceil(N/2)/8) + rb) * 4352.  Rows >= N and columns >= K count as trit 0 with
+                   scales 0.  A tile is 8 chunks of 512 bytes, then 32 scale quads of 8 bytes.  Chunk c holds,
+                   for l = 4 g + t (g = 0..7 the row pair within the tile, t = 0..3), 16 bytes at 512 c + 16 l:
+                   four little-endian words (s, h), s = 0, 1, h = 0, 1, at byte 8 s + 4 h; byte e of word (s, h)
+                   is the column byte (as in format 2: code(2p, plane 1) | code(2p, plane 2) << 2 |
+                   code(2p+1, plane 1) << 4 | code(2p+1, plane 2) << 6) of row pair p = 8 rb + g and column
+                   512 sb + 128 (2 h + t // 2) + 8 (2 c + s) + 4 (t % 2) + e.  Scale quad l = 4 g + t at byte
+                   4096 + 8 l: alpha1[2p], alpha2[2p], alpha1[2p+1], alpha2[2p+1] (u16 each) of group 4 sb + t.
+
 Written independently of the CUDA pack/unpack kernels (plain numpy bit operations) so that the two
 can be compared byte for byte.
 """
@@ -227,3 +241,106 @@ def unpack_reference_v2(blob):
     a2 = np.zeros((2 * nrp, K // 128), dtype=np.uint16)
     a1[0::2], a2[0::2], a1[1::2], a2[1::2] = quads[:, :, 0], quads[:, :, 1], quads[:, :, 2], quads[:, :, 3]
     return planes[0], planes[1], a1[:N].view(np.float16), a2[:N].view(np.float16)
+
+
+# ----------------------------------------------------------------------------- format 3
+TILE_V3 = 4352
+
+
+def layout_v3(N, K):
+    if N <= 0 or K <= 0 or K % 128:
+        raise ValueError("N > 0 and K a positive multiple of 128 required")
+    nrp = (N + 1) // 2
+    nrb = (nrp + 7) // 8
+    sbs = (K + 511) // 512
+    return dict(N=N, K=K, nrp=nrp, nrb=nrb, sbs=sbs, codes_off=HEADER_BYTES,
+                total=HEADER_BYTES + nrb * sbs * TILE_V3)
+
+
+def _tile_maps_v3():
+    """For every code byte of a tile: (row pair within the tile, column within the superblock); for every scale
+    quad: (row pair within the tile, group within the superblock).  Written out from the format description."""
+    rp = np.zeros(4096, dtype=np.int64)
+    col = np.zeros(4096, dtype=np.int64)
+    for c in range(8):
+        for g in range(8):
+            for t in range(4):
+                for s in range(2):
+                    for h in range(2):
+                        for e in range(4):
+                            b = 512 * c + 16 * (4 * g + t) + 8 * s + 4 * h + e
+                            rp[b] = g
+                            col[b] = 128 * (2 * h + t // 2) + 8 * (2 * c + s) + 4 * (t % 2) + e
+    qrp = np.repeat(np.arange(8), 4)
+    qgrp = np.tile(np.arange(4), 8)
+    return rp, col, qrp, qgrp
+
+
+def pack_reference_v3(T1, T2, alpha1, alpha2):
+    """Planes int8 [N,K], scales fp16 [N,K/128] -> format-3 blob (numpy uint8)."""
+    T1 = np.asarray(T1, dtype=np.int8)
+    T2 = np.asarray(T2, dtype=np.int8)
+    N, K = T1.shape
+    L = layout_v3(N, K)
+    if np.any(np.abs(T1) > 1) or np.any(np.abs(T2) > 1):
+        raise ValueError("trit out of range")
+    nrb, sbs = L["nrb"], L["sbs"]
+    rows, cols = 16 * nrb, 512 * sbs
+    q = np.ones((2, rows, cols), dtype=np.uint8)                   # [plane, row, column]; padding is trit 0
+    q[0, :N, :K] = (T1.astype(np.int16) + 1).astype(np.uint8)
+    q[1, :N, :K] = (T2.astype(np.int16) + 1).astype(np.uint8)
+    col_byte = (q[0, 0::2] | (q[1, 0::2] << 2) | (q[0, 1::2] << 4) | (q[1, 1::2] << 6)).astype(np.uint8)
+    sc = np.zeros((rows, 4 * sbs, 2), dtype="<u2")                 # [row, group, plane]
+    sc[:N, :K // 128, 0] = np.asarray(alpha1, dtype=np.float16).view(np.uint16)
+    sc[:N, :K // 128, 1] = np.asarray(alpha2, dtype=np.float16).view(np.uint16)
+    quads = np.concatenate([sc[0::2], sc[1::2]], axis=2)           # [row pair, group, 4]
+    blob = np.zeros(L["total"], dtype=np.uint8)
+    hdr = MAGIC + struct.pack("<IIiiiiQQQ", 1, 3, N, K, 128, 512 * sbs, L["codes_off"], TILE_V3, L["total"])
+    blob[:len(hdr)] = np.frombuffer(hdr, dtype=np.uint8)
+    rp, col, qrp, qgrp = _tile_maps_v3()
+    for sb in range(sbs):
+        for rb in range(nrb):
+            off = HEADER_BYTES + (sb * nrb + rb) * TILE_V3
+            blob[off:off + 4096] = col_byte[8 * rb + rp, 512 * sb + col]
+            blob[off + 4096:off + TILE_V3] = np.ascontiguousarray(quads[8 * rb + qrp, 4 * sb + qgrp]).reshape(-1).view(np.uint8)
+    return blob
+
+
+def unpack_reference_v3(blob):
+    """Format-3 blob (numpy uint8) -> T1, T2 int8 [N,K], alpha1, alpha2 fp16 [N,K/128]."""
+    blob = np.asarray(blob, dtype=np.uint8)
+    hdr = bytes(blob[:HEADER_BYTES])
+    if hdr[:8] != MAGIC:
+        raise ValueError("bad magic")
+    version, fmt, N, K, group, K_pad, codes_off, tile, total = struct.unpack("<IIiiiiQQQ", hdr[8:56])
+    if version != 1 or fmt != 3 or group != 128 or any(hdr[56:]):
+        raise ValueError("bad version/format/group")
+    L = layout_v3(N, K)
+    if (K_pad, codes_off, tile, total) != (512 * L["sbs"], L["codes_off"], TILE_V3, L["total"]):
+        raise ValueError("header inconsistent with its shape")
+    if blob.size < L["total"]:
+        raise ValueError("blob too small")
+    nrb, sbs = L["nrb"], L["sbs"]
+    col_byte = np.zeros((8 * nrb, 512 * sbs), dtype=np.uint8)
+    quads = np.zeros((8 * nrb, 4 * sbs, 4), dtype="<u2")
+    rp, col, qrp, qgrp = _tile_maps_v3()
+    for sb in range(sbs):
+        for rb in range(nrb):
+            off = HEADER_BYTES + (sb * nrb + rb) * TILE_V3
+            col_byte[8 * rb + rp, 512 * sb + col] = blob[off:off + 4096]
+            quads[8 * rb + qrp, 4 * sb + qgrp] = blob[off + 4096:off + TILE_V3].view("<u2").reshape(32, 4)
+    t = np.zeros((2, 16 * nrb, 512 * sbs), dtype=np.int16)
+    for plane in range(2):
+        for r in range(2):
+            code = (col_byte >> (4 * r + 2 * plane)) & 3
+            if np.any(code == 3):
+                raise ValueError("code 3 found")
+            t[plane, r::2] = code.astype(np.int16) - 1
+    if np.any(t[:, N:] != 0) or np.any(t[:, :, K:] != 0):
+        raise ValueError("padding rows and columns must hold trit 0")
+    a = np.zeros((2, 16 * nrb, 4 * sbs), dtype=np.uint16)
+    a[0, 0::2], a[1, 0::2], a[0, 1::2], a[1, 1::2] = quads[:, :, 0], quads[:, :, 1], quads[:, :, 2], quads[:, :, 3]
+    if np.any(a[:, N:] != 0) or np.any(a[:, :, K // 128:] != 0):
+        raise ValueError("padding scales must be zero")
+    return (t[0, :N, :K].astype(np.int8), t[1, :N, :K].astype(np.int8),
+            np.ascontiguousarray(a[0, :N, :K // 128]).view(np.float16), np.ascontiguousarray(a[1, :N, :K // 128]).view(np.float16))

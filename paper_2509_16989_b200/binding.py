@@ -14,6 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libptqtp.so")
 GROUP = 128
 FORMAT_V1 = 1
 FORMAT_V2 = 2
+FORMAT_V3 = 3
 DEFAULT_FORMAT = FORMAT_V2
 HEADER_BYTES = 256
 MAX_BATCH = 64
@@ -24,7 +25,8 @@ OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_SIZE, ERR_TRIT, ERR_FORMAT, ERR_CUDA, ER
 EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny",
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
            "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws",
-           "ptqtp_gemm_skinny_static", "ptqtp_kernel_status", "ptqtp_gemv_swiglu")
+           "ptqtp_gemm_skinny_static", "ptqtp_kernel_status", "ptqtp_gemv_swiglu", "ptqtp_kernel_status_clear",
+           "ptqtp_set_wait_limit", "ptqtp_test_fail_next_wait")
 
 
 class PtqtpError(RuntimeError):
@@ -84,6 +86,12 @@ def lib():
         L.ptqtp_kernel_status.argtypes = [ctypes.POINTER(ctypes.c_int32), vp]
         L.ptqtp_set_overlap.restype = ctypes.c_int
         L.ptqtp_set_overlap.argtypes = [ctypes.c_int]
+        L.ptqtp_kernel_status_clear.restype = ctypes.c_int
+        L.ptqtp_kernel_status_clear.argtypes = [vp]
+        L.ptqtp_set_wait_limit.restype = ctypes.c_int
+        L.ptqtp_set_wait_limit.argtypes = [ctypes.c_int]
+        L.ptqtp_test_fail_next_wait.restype = None
+        L.ptqtp_test_fail_next_wait.argtypes = [ctypes.c_int]
         _lib = L
     return _lib
 
@@ -180,9 +188,9 @@ def ptqtp_gemv_cfg(packed, N, K, x, y=None, rows_per_warp=0, k_split=0, ctas_per
     return y
 
 
-def ptqtp_gemv_swiglu(packed, N, K, x, y=None, stream=None):
-    """y[N/2] = silu(row 2i) * row 2i+1 of the layer applied to x; packed holds gate/up rows interleaved (format 2)."""
-    shape = make_shape(N, K, fmt=FORMAT_V2)
+def ptqtp_gemv_swiglu(packed, N, K, x, y=None, stream=None, fmt=FORMAT_V2):
+    """y[N/2] = silu(row 2i) * row 2i+1 of the layer applied to x; packed holds gate/up rows interleaved (format 2 or 3)."""
+    shape = make_shape(N, K, fmt=fmt)
     if y is None:
         y = torch.empty(N // 2, dtype=torch.float16, device=x.device)
     st = lib().ptqtp_gemv_swiglu(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
@@ -264,9 +272,24 @@ def ptqtp_kernel_status(stream=None):
     return int(out.value)
 
 
+def ptqtp_kernel_status_clear(stream=None):
+    """Reset the device-side health word to 0 (enqueued on the stream)."""
+    _check(lib().ptqtp_kernel_status_clear(_stream_ptr(stream)), "ptqtp_kernel_status_clear")
+
+
+def ptqtp_set_wait_limit(polls):
+    """Polls after which a bounded wait for a bulk copy gives up; returns the old value."""
+    return int(lib().ptqtp_set_wait_limit(int(polls)))
+
+
+def ptqtp_test_fail_next_wait(launches):
+    """Test hook: the next `launches` format-3 batch-1 launches let one bounded wait run out."""
+    lib().ptqtp_test_fail_next_wait(int(launches))
+
+
 def ptqtp_set_overlap(level):
-    """Overlap level of consecutive GEMV calls: 0 off, 1 programmatic dependent launch, 2 (default) also the
-    speculative read of x.  True/False mean 2/0.  Returns the old level."""
+    """Overlap level of consecutive GEMV calls: 0 (default) plain launches, 1 programmatic dependent launch, 2 also
+    the speculative read of x.  True/False mean 2/0.  Returns the old level."""
     if level is True:
         level = 2
     return int(lib().ptqtp_set_overlap(int(level)))

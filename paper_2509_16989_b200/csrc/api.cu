@@ -1,5 +1,6 @@
 // C ABI of libptqtp: argument validation and dispatch.  Declarations and contracts: include/ptqtp.h.
 #include <string.h>
+#include <atomic>
 #include <mutex>
 #include <vector>
 #include "ptqtp_internal.h"
@@ -7,9 +8,19 @@
 namespace ptqtp {
 
 static thread_local int g_last_cuda_error = 0;
-static int g_overlap = 2;
+// Process-wide settings, read by every launch and written by their setters from any thread.
+static std::atomic<int> g_overlap{0};                  // ptqtp_set_overlap: plain launches unless the caller opts in
+static std::atomic<int> g_wait_limit{1 << 22};         // ptqtp_set_wait_limit
+static std::atomic<int> g_fail_waits{0};               // ptqtp_test_fail_next_wait
 
-bool overlap_enabled() { return g_overlap != 0; }
+bool overlap_enabled() { return g_overlap.load(std::memory_order_relaxed) != 0; }
+int wait_poll_limit() { return g_wait_limit.load(std::memory_order_relaxed); }
+bool take_injected_wait_failure() {
+    int n = g_fail_waits.load(std::memory_order_relaxed);
+    while (n > 0)
+        if (g_fail_waits.compare_exchange_weak(n, n - 1)) return true;
+    return false;
+}
 
 // Streams on which ptqtp_pack was the library's last call: the next GEMV launch there is a plain launch, so that
 // it reads the packed planes only after the pack kernel has completed (a dependent launch reads them earlier).
@@ -37,7 +48,7 @@ bool consume_pack(cudaStream_t st) {
     }
     return false;
 }
-bool speculation_enabled() { return g_overlap >= 2; }
+bool speculation_enabled() { return g_overlap.load(std::memory_order_relaxed) >= 2; }
 
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = (int)e; }
 
@@ -66,16 +77,18 @@ int sm_count() {
 
 // Layout of either format, as selected by shape->format.
 struct AnyLayout {
-    bool v2;
+    bool v2, v3;
     Layout l1;
     Layout2 l2;
+    Layout3 l3;
 };
 
 static ptqtp_status check_packed(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, AnyLayout* L) {
     if (!shape || !packed) return PTQTP_ERR_NULL;
     if (!shape_ok(shape)) return PTQTP_ERR_SHAPE;
     L->v2 = shape->format == PTQTP_FORMAT_V2;
-    if (L->v2) L->l2 = make_layout2(shape); else L->l1 = make_layout(shape);
+    L->v3 = shape->format == PTQTP_FORMAT_V3;
+    if (L->v3) L->l3 = make_layout3(shape); else if (L->v2) L->l2 = make_layout2(shape); else L->l1 = make_layout(shape);
     if (!aligned16(packed)) return PTQTP_ERR_ALIGN;
     if (packed_bytes < packed_total(shape)) return PTQTP_ERR_SIZE;
     return PTQTP_OK;
@@ -85,6 +98,10 @@ static int default_gemv_arith() { return 3; }
 
 static ptqtp_status gemv_any(const AnyLayout& L, const void* packed, const uint16_t* x, uint16_t* y, int p0, int p1,
                              int p2, int p3, int p4, cudaStream_t st) {
+    if (L.v3) {
+        if (p4 != -1 && p4 != 5) return PTQTP_ERR_CONFIG;
+        return launch_gemv4(L.l3, packed, x, y, p1, p2, p3, p0, st);
+    }
     if (L.v2) {
         if ((p4 != -1 && p4 != 3 && p4 != 4) || (p0 != 0 && p4 == 4)) return PTQTP_ERR_CONFIG;
         if (p4 == 4) {                       // tensor-core kernel
@@ -123,7 +140,8 @@ ptqtp_status ptqtp_pack(const ptqtp_shape* shape, const int8_t* T1, const int8_t
     if (dev_status && (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return PTQTP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     note_pack(st);
-    return L.v2 ? launch_pack2(L.l2, T1, T2, alpha1, alpha2, packed, dev_status, st)
+    return L.v3 ? launch_pack3(L.l3, T1, T2, alpha1, alpha2, packed, dev_status, st)
+         : L.v2 ? launch_pack2(L.l2, T1, T2, alpha1, alpha2, packed, dev_status, st)
                 : launch_pack(L.l1, T1, T2, alpha1, alpha2, packed, dev_status, st);
 }
 
@@ -136,7 +154,8 @@ ptqtp_status ptqtp_unpack(const ptqtp_shape* shape, const void* packed, size_t p
     if (!aligned16(T1) || !aligned16(T2) || !aligned16(alpha1) || !aligned16(alpha2)) return PTQTP_ERR_ALIGN;
     if (dev_status && (reinterpret_cast<uintptr_t>(dev_status) & 3u)) return PTQTP_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return L.v2 ? launch_unpack2(L.l2, packed, T1, T2, alpha1, alpha2, dev_status, st)
+    return L.v3 ? launch_unpack3(L.l3, packed, T1, T2, alpha1, alpha2, dev_status, st)
+         : L.v2 ? launch_unpack2(L.l2, packed, T1, T2, alpha1, alpha2, dev_status, st)
                 : launch_unpack(L.l1, packed, T1, T2, alpha1, alpha2, dev_status, st);
 }
 
@@ -148,7 +167,8 @@ ptqtp_status ptqtp_gemv_cfg(const ptqtp_shape* shape, const void* packed, size_t
     ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
     if (s != PTQTP_OK) return s;
     if (!aligned16(x) || !aligned16(y)) return PTQTP_ERR_ALIGN;
-    if (rows_per_warp < 0 || k_split < 0 || ctas_per_sm < 0 || depth < 0 || arith < -1) return PTQTP_ERR_CONFIG;
+    if (rows_per_warp < 0 || k_split < -1 || ctas_per_sm < 0 || depth < 0 || arith < -1) return PTQTP_ERR_CONFIG;
+    if (k_split < 0 && !L.v2 && !L.v3) return PTQTP_ERR_CONFIG;
     return gemv_any(L, packed, x, y, rows_per_warp, k_split, ctas_per_sm, depth, arith,
                     static_cast<cudaStream_t>(stream));
 }
@@ -164,9 +184,10 @@ ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape* shape, const void* packed, siz
     AnyLayout L;
     ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
     if (s != PTQTP_OK) return s;
-    if (!L.v2) return PTQTP_ERR_CONFIG;
+    if (!L.v2 && !L.v3) return PTQTP_ERR_CONFIG;
     if (shape->n_out % 2) return PTQTP_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(y)) return PTQTP_ERR_ALIGN;
+    if (L.v3) return launch_gemv4(L.l3, packed, x, y, 0, 0, 0, 0, static_cast<cudaStream_t>(stream), true);
     return launch_gemv2(L.l2, packed, x, y, 0, 0, 0, 0, static_cast<cudaStream_t>(stream), true);
 }
 
@@ -200,7 +221,9 @@ ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, siz
         }
         return launch_gemv2(L.l2, packed, X, Y, 0, 0, 0, 0, st);
     }
-    return launch_gemm_skinny(L.l1, packed, m, X, Y, st);
+    // formats 1 and 3 are batch-1 layouts: the small-batch kernels read format 2
+    if (m != 1) return PTQTP_ERR_CONFIG;
+    return gemv_any(L, packed, X, Y, 0, 0, 0, 0, -1, st);
 }
 
 size_t ptqtp_gemm_skinny_workspace_size(const ptqtp_shape* shape, int32_t m) {
@@ -253,7 +276,7 @@ ptqtp_status ptqtp_gemv_host(const ptqtp_shape* shape, const void* packed, size_
     // the kernel stores y there itself and the copy back is saved; otherwise y goes through y_dev.
     uint16_t* y_target = y_dev;
     bool direct = false;
-    if (L.v2 && aligned16(y_host)) {
+    if ((L.v2 || L.v3) && aligned16(y_host)) {
         cudaPointerAttributes attr;
         if (cudaPointerGetAttributes(&attr, y_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
             attr.devicePointer != nullptr) {
@@ -264,7 +287,8 @@ ptqtp_status ptqtp_gemv_host(const ptqtp_shape* shape, const void* packed, size_
         }
     }
     // between its two copies the kernel never overlaps another GEMV: it gets whole SMs
-    s = L.v2 ? launch_gemv2(L.l2, packed, x_dev, y_target, -1, 0, 0, 0, st)
+    s = L.v3 ? launch_gemv4(L.l3, packed, x_dev, y_target, -1, 0, 0, 0, st)
+      : L.v2 ? launch_gemv2(L.l2, packed, x_dev, y_target, -1, 0, 0, 0, st)
              : gemv_any(L, packed, x_dev, y_dev, 0, 0, 0, 0, -1, st);
     if (s != PTQTP_OK) return s;
     if (!direct) {
@@ -280,13 +304,18 @@ ptqtp_status ptqtp_parse_header(const void* header_host, size_t bytes, ptqtp_sha
     Header h;
     memcpy(&h, header_host, sizeof(Header));
     if (memcmp(h.magic, "PTQTPB2\0", 8) != 0 || h.version != kVersion ||
-        (h.format != PTQTP_FORMAT_V1 && h.format != PTQTP_FORMAT_V2))
+        (h.format != PTQTP_FORMAT_V1 && h.format != PTQTP_FORMAT_V2 && h.format != PTQTP_FORMAT_V3))
         return PTQTP_ERR_FORMAT;
     ptqtp_shape s = {h.n, h.k, h.group, (int32_t)h.format};
     if (!shape_ok(&s)) return PTQTP_ERR_FORMAT;
     if (h.format == PTQTP_FORMAT_V1) {
         const Layout L = make_layout(&s);
         if (h.k_pad != L.k_pad || h.codes_off != L.codes_off || h.scales_off != L.scales_off || h.total != L.total)
+            return PTQTP_ERR_FORMAT;
+    } else if (h.format == PTQTP_FORMAT_V3) {
+        const Layout3 L = make_layout3(&s);
+        if (h.k_pad != L.sbs * kSuper3 || h.codes_off != L.codes_off || h.scales_off != (uint64_t)kTile3 ||
+            h.total != L.total)
             return PTQTP_ERR_FORMAT;
     } else {
         const Layout2 L = make_layout2(&s);
@@ -320,10 +349,25 @@ ptqtp_status ptqtp_kernel_status(int32_t* status_host, void* stream) {
     return copy_gemv2_status(status_host, static_cast<cudaStream_t>(stream));
 }
 
-int ptqtp_set_overlap(int enabled) {
-    const int old = g_overlap;
-    g_overlap = enabled <= 0 ? 0 : enabled >= 2 ? 2 : 1;
-    return old;
+ptqtp_status ptqtp_kernel_status_clear(void* stream) {
+    int* word = nullptr;
+    ptqtp_status s = gemv_status_word(&word);
+    if (s != PTQTP_OK) return s;
+    cudaError_t e = cudaMemsetAsync(word, 0, sizeof(int), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
+    return PTQTP_OK;
+}
+
+int ptqtp_set_overlap(int level) {
+    return g_overlap.exchange(level <= 0 ? 0 : level >= 2 ? 2 : 1);
+}
+
+int ptqtp_set_wait_limit(int polls) {
+    return g_wait_limit.exchange(polls < 1 ? 1 : polls);
+}
+
+void ptqtp_test_fail_next_wait(int launches) {
+    g_fail_waits.store(launches < 0 ? 0 : launches);
 }
 
 int ptqtp_version(void) { return 100; }

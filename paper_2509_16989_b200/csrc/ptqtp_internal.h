@@ -30,7 +30,7 @@ static_assert(sizeof(Header) <= PTQTP_HEADER_BYTES, "header must fit its slot");
 
 inline bool shape_ok(const ptqtp_shape* s) {
     return s && s->n_out > 0 && s->k_in > 0 && s->group == kGroup && s->k_in % kGroup == 0 &&
-           (s->format == PTQTP_FORMAT_V1 || s->format == PTQTP_FORMAT_V2);
+           (s->format == PTQTP_FORMAT_V1 || s->format == PTQTP_FORMAT_V2 || s->format == PTQTP_FORMAT_V3);
 }
 
 inline Layout make_layout(const ptqtp_shape* s) {
@@ -81,8 +81,40 @@ __host__ __device__ inline size_t unit_offset(const Layout2& L, int rp, int s) {
     return (size_t)s * L.nrp * kUnit2 + (size_t)rp * (s == L.slices - 1 ? L.last_unit : kUnit2);
 }
 
+// ---- format 3: tiles of 8 row pairs x 512 columns in tensor-core fragment order (see ptqtp.h) ----
+constexpr int kSuper3 = 512;         // input columns per tile (four scale groups)
+constexpr int kTileRp3 = 8;          // row pairs per tile
+constexpr int kTileCodes3 = 4096;    // code bytes of a tile
+constexpr int kTile3 = 4352;         // bytes of a tile: 4096 code bytes + 32 scale quads of 8 bytes
+
+struct Layout3 {
+    int n, k, nrp;                   // rows, columns, row pairs = ceil(n / 2)
+    int nrb;                         // row blocks = ceil(nrp / 8)
+    int sbs;                         // superblocks = ceil(k / 512)
+    size_t codes_off, total;
+};
+
+inline Layout3 make_layout3(const ptqtp_shape* s) {
+    Layout3 L;
+    L.n = s->n_out;
+    L.k = s->k_in;
+    L.nrp = (s->n_out + 1) / 2;
+    L.nrb = (L.nrp + kTileRp3 - 1) / kTileRp3;
+    L.sbs = (s->k_in + kSuper3 - 1) / kSuper3;
+    L.codes_off = PTQTP_HEADER_BYTES;
+    L.total = L.codes_off + (size_t)L.nrb * L.sbs * kTile3;
+    return L;
+}
+
+// Byte offset (from codes_off) of tile (superblock sb, row block rb): superblock-major, so the tiles of one
+// superblock for consecutive row blocks are contiguous.
+__host__ __device__ inline size_t tile_offset3(const Layout3& L, int rb, int sb) {
+    return ((size_t)sb * L.nrb + rb) * kTile3;
+}
+
 inline size_t packed_total(const ptqtp_shape* s) {
-    return s->format == PTQTP_FORMAT_V2 ? make_layout2(s).total : make_layout(s).total;
+    return s->format == PTQTP_FORMAT_V3 ? make_layout3(s).total
+         : s->format == PTQTP_FORMAT_V2 ? make_layout2(s).total : make_layout(s).total;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -97,13 +129,18 @@ ptqtp_status launch_unpack(const Layout& L, const void* packed, int8_t* T1, int8
                            uint16_t* a2, int32_t* dev_status, cudaStream_t st);
 ptqtp_status launch_gemv(const Layout& L, const void* packed, const uint16_t* x, uint16_t* y,
                          int rows_per_warp, int k_split, int ctas_per_sm, int depth, int arith, cudaStream_t st);
-ptqtp_status launch_gemm_skinny(const Layout& L, const void* packed, int m, const uint16_t* X,
-                                uint16_t* Y, cudaStream_t st);
 ptqtp_status launch_pack2(const Layout2& L, const int8_t* T1, const int8_t* T2, const uint16_t* a1,
                           const uint16_t* a2, void* packed, int32_t* dev_status, cudaStream_t st);
 ptqtp_status launch_unpack2(const Layout2& L, const void* packed, int8_t* T1, int8_t* T2, uint16_t* a1,
                             uint16_t* a2, int32_t* dev_status, cudaStream_t st);
 ptqtp_status launch_gemv2(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
+                          int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated = false);
+ptqtp_status launch_pack3(const Layout3& L, const int8_t* T1, const int8_t* T2, const uint16_t* a1,
+                          const uint16_t* a2, void* packed, int32_t* dev_status, cudaStream_t st);
+ptqtp_status launch_unpack3(const Layout3& L, const void* packed, int8_t* T1, int8_t* T2, uint16_t* a1,
+                            uint16_t* a2, int32_t* dev_status, cudaStream_t st);
+// warps: per CTA (0 = library choice, -1 = as many as fit); depth: tiles in flight per warp (0 = library choice)
+ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
                           int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated = false);
 size_t skinny3_workspace_bytes(int k, int m);
 ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, void* workspace,
@@ -117,6 +154,8 @@ ptqtp_status launch_gemv3(const Layout2& L, const void* packed, int m, const uin
 int sm_count();
 bool speculation_enabled();       // speculative read of x before the dependency wait (ptqtp_set_overlap(2))
 bool overlap_enabled();           // programmatic dependent launch of the GEMV kernels (ptqtp_set_overlap)
+int wait_poll_limit();            // polls of an mbarrier before a bounded wait gives up (ptqtp_set_wait_limit)
+bool take_injected_wait_failure();   // test hook: true once per armed failure (ptqtp_test_fail_next_wait)
 bool consume_pack(cudaStream_t st);   // true once after ptqtp_pack on this stream: the next GEMV launch is plain
 
 }  // namespace ptqtp

@@ -14,7 +14,7 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-FORMATS = (binding.FORMAT_V1, binding.FORMAT_V2)
+FORMATS = (binding.FORMAT_V1, binding.FORMAT_V2, binding.FORMAT_V3)
 
 
 def pack_case(c, fmt=None):

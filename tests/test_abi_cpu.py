@@ -36,7 +36,7 @@ def test_every_declared_symbol_is_exported(L):
 
 def test_packed_size_is_memory_formula_plus_header_and_padding(L):
     for N, K in ((3072, 1024), (4096, 4096), (1024, 4096), (14336, 4096), (4096, 14336), (8192, 28672)):
-        for fmt, lay in ((1, pf.layout), (2, pf.layout_v2)):
+        for fmt, lay in ((1, pf.layout), (2, pf.layout_v2), (3, pf.layout_v3)):
             got = binding.packed_size(N, K, fmt=fmt)
             assert got == lay(N, K)["total"]
             assert got == pf.HEADER_BYTES + pf.memory_formula_bits(N, K) // 8      # no padding at these shapes
@@ -45,10 +45,13 @@ def test_packed_size_is_memory_formula_plus_header_and_padding(L):
     # format 2: an odd N stores one more row; a unit whose size is not a multiple of 16 is padded
     assert binding.packed_size(7, 1152, fmt=2) == 256 + 4 * (1152 + 72 + 8) == pf.layout_v2(7, 1152)["total"]
     assert binding.packed_size(3, 4224, fmt=2) == 256 + 2 * (2176 * 2 + 128 + 8 + 8) == pf.layout_v2(3, 4224)["total"]
+    # format 3: whole tiles of 16 rows x 512 columns, 4352 bytes each
+    assert binding.packed_size(7, 1152, fmt=3) == 256 + 1 * 3 * 4352 == pf.layout_v3(7, 1152)["total"]
+    assert binding.packed_size(33, 512, fmt=3) == 256 + 3 * 1 * 4352 == pf.layout_v3(33, 512)["total"]
     for bad in ((0, 128), (4, 0), (4, 100), (-1, 128)):
         assert binding.packed_size(*bad) == 0
     assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 64, 1))) == 0
-    assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 128, 3))) == 0
+    assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 128, 4))) == 0
     assert L.ptqtp_packed_size(ctypes.byref(binding.Shape(4, 128, 128, 0))) == 0
 
 
@@ -60,6 +63,12 @@ def test_parse_header_accepts_reference_blob_and_rejects_damage(L):
     bad2[40] ^= 8         # bytes per row pair no longer match the shape
     with pytest.raises(binding.PtqtpError):
         binding.ptqtp_parse_header(bytes(bad2))
+    blob3 = pf.pack_reference_v3(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+    assert binding.ptqtp_parse_header(bytes(blob3[:256])) == (3, 1152, 3)
+    bad3 = blob3[:256].copy()
+    bad3[40] ^= 8         # bytes per tile no longer 4352
+    with pytest.raises(binding.PtqtpError):
+        binding.ptqtp_parse_header(bytes(bad3))
     blob = pf.pack_reference(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
     assert binding.ptqtp_parse_header(bytes(blob[:256])) == (3, 1152, 1)
     bad = blob[:256].copy()
@@ -105,6 +114,24 @@ def test_host_side_validation_codes(L):
     v1 = binding.make_shape(8, 256, fmt=binding.FORMAT_V1)
     assert L.ptqtp_gemv_swiglu(ctypes.byref(v1), ok_ptr, binding.packed_size(8, 256, fmt=binding.FORMAT_V1), ok_ptr, ok_ptr,
                                None) == binding.ERR_CONFIG
+    # formats 1 and 3 are batch-1 layouts: the small-batch calls refuse them for M > 1
+    for fmt in (binding.FORMAT_V1, binding.FORMAT_V3):
+        sh = binding.make_shape(8, 256, fmt=fmt)
+        sz = binding.packed_size(8, 256, fmt=fmt)
+        assert L.ptqtp_gemm_skinny(ctypes.byref(sh), ok_ptr, sz, 2, ok_ptr, ok_ptr, None) == binding.ERR_CONFIG
+        assert L.ptqtp_gemm_skinny_ws(ctypes.byref(sh), ok_ptr, sz, 2, ok_ptr, ok_ptr, ok_ptr, 1 << 20, None) == binding.ERR_CONFIG
+        assert L.ptqtp_gemm_skinny_workspace_size(ctypes.byref(sh), 2) == 0
+
+
+def test_process_wide_settings_defaults_and_setters(L):
+    # plain launches are the default: every buffer, the packed blob included, follows stream order
+    assert L.ptqtp_set_overlap(1) == 0
+    assert L.ptqtp_set_overlap(7) == 1
+    assert L.ptqtp_set_overlap(-3) == 2
+    assert L.ptqtp_set_overlap(0) == 0
+    assert L.ptqtp_set_wait_limit(1000) == 1 << 22
+    assert L.ptqtp_set_wait_limit(0) == 1000
+    assert L.ptqtp_set_wait_limit(1 << 22) == 1
 
 
 def test_status_strings(L):
@@ -160,6 +187,47 @@ def test_reference_format2_roundtrip_layout_and_damage_detection():
     bad[tail + 140] = 1
     with pytest.raises(ValueError):
         pf.unpack_reference_v2(bad)
+
+
+def test_reference_format3_roundtrip_layout_and_damage_detection():
+    c = make_case(21, 1152, seed=4)                      # 11 row pairs -> 2 row blocks; 1152 columns -> 3 superblocks
+    blob = pf.pack_reference_v3(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+    t1, t2, a1, a2 = pf.unpack_reference_v3(blob)
+    assert np.array_equal(t1, c["T1"]) and np.array_equal(t2, c["T2"])
+    assert np.array_equal(a1.view(np.uint16), c["alpha1"].view(np.uint16))
+    assert np.array_equal(a2.view(np.uint16), c["alpha2"].view(np.uint16))
+    assert blob.size == 256 + 2 * 3 * 4352
+
+    def column_byte(rp, col):
+        return ((int(c["T1"][2 * rp, col]) + 1) | (int(c["T2"][2 * rp, col]) + 1) << 2
+                | (int(c["T1"][2 * rp + 1, col]) + 1) << 4 | (int(c["T2"][2 * rp + 1, col]) + 1) << 6)
+
+    # One byte by hand: row pair 9 (rows 18, 19) = row block 1, g = 1; column 700 = superblock 1, column 188 of it:
+    # group 1 (h = 0, t / 2 = 1), column 60 of the group = k-step 7 (chunk 3, s = 1), second half (t % 2 = 1), e = 0
+    # -> t = 3, lane 4 * 1 + 3 = 7, byte 512 * 3 + 16 * 7 + 8 * 1 + 4 * 0 + 0 of tile (sb 1, rb 1) = tile number 1 * 2 + 1
+    off = 256 + 3 * 4352 + 512 * 3 + 16 * 7 + 8
+    assert int(blob[off]) == column_byte(9, 700)
+    # column 700 + 256 = 956 is group 3 of the same superblock: h = 1, same lane, four bytes further
+    assert int(blob[off + 4]) == column_byte(9, 956)
+    # scale quad of row pair 9, group 5 (superblock 1, t = 1): lane 4 * 1 + 1 = 5 of the same tile
+    q = 256 + 3 * 4352 + 4096 + 8 * 5
+    assert bytes(blob[q:q + 8]) == (c["alpha1"][18, 5].tobytes() + c["alpha2"][18, 5].tobytes()
+                                    + c["alpha1"][19, 5].tobytes() + c["alpha2"][19, 5].tobytes())
+    # row 21 does not exist: row pair 10 (row block 1, g = 2) has trit 0 (code 1) and zero scales in its upper half
+    first = 256 + 1 * 4352 + 16 * (4 * 2 + 0)
+    assert (int(blob[first]) >> 4) == 0b0101
+    assert not blob[256 + 4352 + 4096 + 8 * 8 + 4:256 + 4352 + 4096 + 8 * 8 + 8].any()
+    # columns 1152 .. 1535 of superblock 2 do not exist: group 1 of that superblock (t = 2, 3 with h = 0) holds 0x55
+    pad = 256 + (2 * 2 + 0) * 4352 + 16 * 2
+    assert int(blob[pad]) == 0x55
+    bad = blob.copy()
+    bad[256] |= 3
+    with pytest.raises(ValueError):
+        pf.unpack_reference_v3(bad)
+    bad = blob.copy()
+    bad[pad] = 0x54
+    with pytest.raises(ValueError):
+        pf.unpack_reference_v3(bad)
 
 
 def test_reference_format_roundtrip_and_damage_detection():

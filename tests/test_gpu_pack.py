@@ -11,13 +11,18 @@ from gpu_util import FORMATS, dev
 pytestmark = pytest.mark.gpu
 
 
+WRITERS = {binding.FORMAT_V1: pf.pack_reference, binding.FORMAT_V2: pf.pack_reference_v2,
+           binding.FORMAT_V3: pf.pack_reference_v3}
+READERS = {binding.FORMAT_V1: pf.unpack_reference, binding.FORMAT_V2: pf.unpack_reference_v2,
+           binding.FORMAT_V3: pf.unpack_reference_v3}
+
+
 def reference_blob(c, fmt):
-    writer = pf.pack_reference if fmt == binding.FORMAT_V1 else pf.pack_reference_v2
-    return writer(c["T1"], c["T2"], c["alpha1"], c["alpha2"])
+    return WRITERS[fmt](c["T1"], c["T2"], c["alpha1"], c["alpha2"])
 
 
 def reference_unpack(blob, fmt):
-    return (pf.unpack_reference if fmt == binding.FORMAT_V1 else pf.unpack_reference_v2)(blob)
+    return READERS[fmt](blob)
 
 
 def roundtrip(c, fmt):
@@ -34,7 +39,7 @@ def roundtrip(c, fmt):
 
 @pytest.mark.parametrize("fmt", FORMATS)
 @pytest.mark.parametrize("N,K", [(1, 128), (2, 128), (3, 256), (7, 1152), (33, 2048), (130, 3200), (9, 4224),
-                                 (64, 14336), QWEN3_0P6B_UP])
+                                 (64, 14336), (17, 512), (16, 640), QWEN3_0P6B_UP])
 def test_roundtrip_and_bytes_match_reference_writer(N, K, fmt):
     c = make_case(N, K, seed=N + K)
     blob = roundtrip(c, fmt)
@@ -108,13 +113,15 @@ def test_invalid_trit_sets_device_status_and_kernel_completes(fmt):
 def test_unpack_reports_header_mismatch(fmt):
     c = make_case(8, 1024, seed=10)
     packed, _ = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=fmt)
-    *_, st = binding.ptqtp_unpack(packed, 4, 2048, fmt=fmt)      # same byte size, different shape
+    other_shape = (24, 512) if fmt == binding.FORMAT_V3 else (4, 2048)
+    assert binding.packed_size(*other_shape, fmt=fmt) == packed.numel()
+    *_, st = binding.ptqtp_unpack(packed, *other_shape, fmt=fmt)      # same byte size, different shape
     torch.cuda.synchronize()
     assert int(st.item()) == binding.ERR_FORMAT
-    other = binding.FORMAT_V1 + binding.FORMAT_V2 - fmt
-    if binding.packed_size(8, 1024, fmt=other) <= packed.numel():
-        *_, st = binding.ptqtp_unpack(packed, 8, 1024, fmt=other)    # a blob of the other format
-        assert int(st.item()) == binding.ERR_FORMAT
+    for other in FORMATS:
+        if other != fmt and binding.packed_size(8, 1024, fmt=other) <= packed.numel():
+            *_, st = binding.ptqtp_unpack(packed, 8, 1024, fmt=other)    # a blob of another format
+            assert int(st.item()) == binding.ERR_FORMAT
     packed[0] = 0
     *_, st = binding.ptqtp_unpack(packed, 8, 1024, fmt=fmt)
     assert int(st.item()) == binding.ERR_FORMAT

@@ -1,14 +1,10 @@
 """Realistic-weight stack: 32 layers of LLaMA-3-8B-shaped linears whose planes come from the oracle's
 progressive trit-plane decomposition of W ~ N(0, 0.02^2) with 0.1 % of entries multiplied by 20.
 
-Checks parity of the GEMV on decomposed planes (sampled rows, every matrix type), the reconstruction error
-range, and measures one decode step (224 GEMV calls in one CUDA graph).  One layer is decomposed (the oracle
-needs about 20 s of CPU time per layer); the other 31 are byte copies of its packed blobs at distinct
-addresses, so the step still streams 3.7 GB from HBM.  The measurement is written to gpurun_out/config4.json
-when that directory exists."""
-import json
-import os
-
+Checks parity of the GEMV on decomposed planes (every row, every matrix type), the reconstruction error range,
+and that one decode step (224 GEMV calls in one CUDA graph, replayed) reproduces the results of plain calls bit
+for bit.  One layer is decomposed (the oracle needs about 20 s of CPU time per layer); the other 31 are byte
+copies of its packed blobs at distinct addresses.  The step is timed by `python -m paper_2509_16989_b200.report 4`."""
 import numpy as np
 import pytest
 import torch
@@ -23,7 +19,7 @@ pytestmark = pytest.mark.gpu
 NAMES = ("q", "k", "v", "o", "gate", "up", "down")
 
 
-def test_config4_stack_parity_error_and_time():
+def test_config4_stack_parity_and_error():
     blobs, errs = {}, {}
     for mi, m in enumerate(NAMES):
         N, K = LLAMA3_8B[m]
@@ -37,10 +33,8 @@ def test_config4_stack_parity_error_and_time():
         assert int(st.item()) == 0
         x = make_activations(K, seed=70 + mi)
         y = binding.ptqtp_gemv(packed, N, K, dev(x)).cpu().numpy()
-        rows = np.unique(np.random.default_rng(mi).integers(0, N, 384))
-        ref = layer_fp64_c(d["T1"][rows], d["T2"][rows], d["alpha1_fp16"][rows], d["alpha2_fp16"][rows], x,
-                           threads=max_threads())
-        assert_parity(y[rows], ref, x, m)
+        ref = layer_fp64_c(d["T1"], d["T2"], d["alpha1_fp16"], d["alpha2_fp16"], x, threads=max_threads())
+        assert_parity(y, ref, x, m)
         blobs[m] = packed
         del d, W
     stack = [{m: (blobs[m] if i == 0 else blobs[m].clone()) for m in NAMES} for i in range(32)]
@@ -54,7 +48,6 @@ def test_config4_stack_parity_error_and_time():
                 N, K = LLAMA3_8B[m]
                 binding.ptqtp_gemv(layer[m], N, K, xs[m], y=ys[m], stream=stream)
 
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(stream):
         step()
         stream.synchronize()
@@ -65,23 +58,5 @@ def test_config4_stack_parity_error_and_time():
         for _ in range(3):
             g.replay()
         stream.synchronize()
-        e0.record(stream)
-        for _ in range(20):
-            g.replay()
-        e1.record(stream)
-        stream.synchronize()
-    us = 1e3 * e0.elapsed_time(e1) / 20
     for m in NAMES:                                   # every layer holds the same planes: the last one's result
         assert np.array_equal(ys[m].cpu().numpy().view(np.uint16), first[m].view(np.uint16))
-    nbytes = 32 * sum(N * K // 2 + 4 * N * K // 128 + 2 * K + 2 * N for N, K in (LLAMA3_8B[m] for m in NAMES))
-    result = {"workload": "cfg4 32-layer llama3-8b linear stack, oracle-decomposed weights, batch 1", "calls": 224,
-              "us_per_token": round(us, 1), "gbs": round(nbytes / us / 1e3, 1), "bytes": nbytes,
-              "reconstruction_error": {m: round(float(v), 4) for m, v in errs.items()},
-              "reconstruction_error_mean": round(float(np.mean(list(errs.values()))), 4),
-              "distinct_decomposed_layers": 1}
-    print(json.dumps(result))
-    out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    if os.path.isdir(out):
-        with open(os.path.join(out, "config4.json"), "w") as f:
-            json.dump(result, f)
-    assert us < 5000.0                                # 224 calls; a gross regression guard, not a target

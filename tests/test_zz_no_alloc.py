@@ -3,8 +3,9 @@
 cudaMalloc would stall the device).  Its workspace is a fixed array inside the library.
 
 Checked here through the C ABI: two calls in a row, each against the existing workspace entry point
-(ptqtp_gemm_skinny_ws) on the same inputs, within the parity tolerance of the other GPU tests; sizes beyond the
-fixed array are refused.  The file name makes pytest collect it last."""
+(ptqtp_gemm_skinny_ws) on the same inputs -- within the parity tolerance of the other GPU tests, and, since both
+run the same kernels on the same inputs, bit for bit -- and against the fp64 oracle; sizes beyond the fixed array
+are refused.  The file name makes pytest collect it last."""
 import ctypes
 
 import numpy as np
@@ -13,7 +14,7 @@ import torch
 
 from paper_2509_16989_b200 import binding
 from paper_2509_16989_b200.inputs import make_case
-from gpu_util import REL_L2_TOL, MAX_ABS_COEF, dev
+from gpu_util import REL_L2_TOL, MAX_ABS_COEF, assert_parity, dev, oracle_y
 
 pytestmark = pytest.mark.gpu
 
@@ -53,6 +54,8 @@ def test_static_workspace_entry_point_matches_workspace_entry_point_twice():
         assert rc == binding.OK, binding.status_string(rc)
         torch.cuda.synchronize()
         close_to(Y_new.cpu().numpy(), Y_old.cpu().numpy(), x)
+        assert np.array_equal(Y_new.cpu().numpy().view(np.uint16), Y_old.cpu().numpy().view(np.uint16))
+        assert_parity(Y_new.cpu().numpy(), oracle_y(dict(c, x=x)), x, "static workspace call %d" % call)
 
 
 def test_static_workspace_entry_point_refuses_what_does_not_fit():
