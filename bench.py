@@ -3,7 +3,12 @@
 One step = one pass of the hot path over the seven decode linears of a LLaMA-3-8B layer at
 batch 1 (q, k, v, o, gate, up, down), one ptqtp_gemv call per matrix, on packed planes that are
 already resident in HBM.  Steps rotate over `--sets` distinct copies of the layer (default 8,
-928 MB) so that every packed byte comes from HBM, not from L2.
+928 MB) so that every packed byte comes from HBM, not from L2.  The timed steps are one CUDA graph
+(up to 512 steps per graph), so a run of 20 steps has no graph boundary inside it.
+
+The library's default is plain launches; this program opts in to overlap level 2 (programmatic
+dependent launch with speculative execution) as a decoder would whose packed blobs never change while
+GEMV calls are in flight, and says so in `config.overlap`.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -34,9 +39,13 @@ WORKLOAD = "llama3-8b decode linears (q,k,v,o 4096x4096|1024x4096, gate/up 14336
 MATRICES = ("q", "k", "v", "o", "gate", "up", "down")
 UNIQUE_OF = {"q": "qo", "o": "qo", "k": "kv", "v": "kv", "gate": "gate_up", "up": "gate_up", "down": "down"}
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum over algorithmic bytes in the ncu capture of the 14336x4096 launch of
-# the current GEMV kernel (profiles/gemv2_gate_up_14336x4096.md); set to None when the kernel changes
-DRAM_TRAFFIC_RATIO = 31239424.0 / 31232000.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch in the ncu captures of the current batch-1 kernel, one
+# launch per shape (profiles/gemv4_*.md); None for a shape whose kernel has changed since its capture
+DRAM_TRAFFIC_BYTES = {3: {"qo": None, "kv": None, "gate_up": None, "down": None},
+                      2: {"qo": None, "kv": None, "gate_up": 31239424.0, "down": None}}
+KERNEL_NAME = {2: "gemv2_kernel", 3: "gemv4_kernel"}
+DTYPE = {2: "int16 block-fixed-point x int2 codes -> int32 (dp4a), f32 scale epilogue",
+         3: "int15 block-fixed-point x int2 codes -> int32 (int8 mma), f32 scale epilogue"}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -230,6 +239,39 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- GPU arm
+GRAPH_STEPS = 512            # steps per CUDA graph of the timed run (a 20-step run is one graph)
+
+
+class Chain:
+    """CUDA-graph timing of a list of launch functions on one stream."""
+
+    def __init__(self, torch, stream):
+        self.torch, self.stream = torch, stream
+        self.e0 = torch.cuda.Event(enable_timing=True)
+        self.e1 = torch.cuda.Event(enable_timing=True)
+
+    def capture(self, fn):
+        torch, st = self.torch, self.stream
+        with torch.cuda.stream(st):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                fn()
+            g.replay()                                   # the first replay uploads the graph: part of the set-up
+            st.synchronize()
+        return g
+
+    def time_ms(self, graphs):
+        """Replays the graphs back to back once; device time in ms."""
+        torch, st = self.torch, self.stream
+        with torch.cuda.stream(st):
+            self.e0.record(st)
+            for g in graphs:
+                g.replay()
+            self.e1.record(st)
+            st.synchronize()
+        return self.e0.elapsed_time(self.e1)
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -244,21 +286,29 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=device)
     build.build()
     binding.lib()
+    fmt = args.format
+    # the decode case: packed blobs are immutable while GEMV calls are in flight, so the opt-in overlap applies
+    binding.ptqtp_set_overlap(2)
 
     def dev(a):
         return torch.from_numpy(np.ascontiguousarray(a)).to(device)
 
     cases = make_cases()
     stream = torch.cuda.Stream(device=device)
+    chain = Chain(torch, stream)
     R = args.sets
 
+    def pack_all(f):
+        out = {}
+        for u, c in cases.items():
+            packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=f)
+            torch.cuda.synchronize()
+            assert int(st.item()) == 0
+            out[u] = packed
+        return out
+
     # set 0 is packed from the seeded planes; the other sets are byte copies at distinct addresses
-    base = {}
-    for u, c in cases.items():
-        packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
-        torch.cuda.synchronize()
-        assert int(st.item()) == 0
-        base[u] = packed
+    base = pack_all(fmt)
     sets = []
     for r in range(R):
         sets.append({m: (base[UNIQUE_OF[m]] if (r == 0 and m in ("q", "k", "gate", "down"))
@@ -267,61 +317,30 @@ def run_gpu(args):
     ys = {m: torch.empty(LLAMA3_8B[m][0], dtype=torch.float16, device=device) for m in MATRICES}
     torch.cuda.synchronize()
 
-    def step(r):
+    def step(r, f=fmt, layer_sets=None):
         for m in MATRICES:
             N, K = LLAMA3_8B[m]
-            binding.ptqtp_gemv(sets[r][m], N, K, xs[m], y=ys[m], stream=stream)
+            binding.ptqtp_gemv((layer_sets or sets)[r][m], N, K, xs[m], y=ys[m], stream=stream, fmt=f)
 
-    # warm every buffer once outside any capture, then capture the steps as CUDA graphs
-    for r in range(R):
-        step(r)
+    def steps_fn(k, start=0, **kw):
+        def fn():
+            for i in range(k):
+                step((start + i) % R, **kw)
+        return fn
+
+    # warm every buffer once outside any capture, then capture the timed steps
+    with torch.cuda.stream(stream):
+        steps_fn(R)()
     stream.synchronize()
-    graphs = None
-    big = None
-    huge = None
+    timed_graphs, warm_graphs = None, None
     if not args.no_graph:
-        graphs = []
-        for r in range(R):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                step(r)
-            graphs.append(g)
-        big = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(big, stream=stream):
-            for r in range(R):
-                step(r)
-        # eight rotations in one graph: a graph boundary drains the chain of overlapping launches
-        huge = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(huge, stream=stream):
-            for _ in range(8):
-                for r in range(R):
-                    step(r)
-        # first replays upload the graphs to the device: part of the set-up, like packing the matrices
-        with torch.cuda.stream(stream):
-            for g in graphs + [big, huge]:
-                g.replay()
-        stream.synchronize()
-
-    def run_steps(k, start=0):
-        with torch.cuda.stream(stream):
-            i = 0
-            if graphs is None:
-                while i < k:
-                    step((start + i) % R)
-                    i += 1
-                return
-            while i < k and (start + i) % R != 0:
-                graphs[(start + i) % R].replay()
-                i += 1
-            while k - i >= 8 * R:
-                huge.replay()
-                i += 8 * R
-            while k - i >= R:
-                big.replay()
-                i += R
-            while i < k:
-                graphs[(start + i) % R].replay()
-                i += 1
+        per = min(args.steps, GRAPH_STEPS)
+        full = chain.capture(steps_fn(per))
+        timed_graphs = [full] * (args.steps // per)
+        if args.steps % per:
+            timed_graphs.append(chain.capture(steps_fn(args.steps % per, start=(args.steps // per) * per)))
+        nwarm = max(args.warmup, 3)
+        warm_graphs = [chain.capture(steps_fn(min(nwarm, GRAPH_STEPS)))] * -(-nwarm // GRAPH_STEPS)
 
     def barrier():
         if world > 1:
@@ -330,32 +349,58 @@ def run_gpu(args):
     sampler = ClockSampler(local)
     sampler.start()
 
-    run_steps(max(args.warmup, 3))
+    if timed_graphs is None:
+        with torch.cuda.stream(stream):
+            steps_fn(max(args.warmup, 3))()
+    else:
+        chain.time_ms(warm_graphs)
     stream.synchronize()
-    e0 = torch.cuda.Event(enable_timing=True)
-    e1 = torch.cuda.Event(enable_timing=True)
     barrier()
     torch.cuda.synchronize()
     t_begin = time.perf_counter()
-    e0.record(stream)
-    run_steps(args.steps)
-    e1.record(stream)
-    sampler.sample_now()                                 # the GPU is still working on the enqueued steps
-    stream.synchronize()
+    if timed_graphs is None:
+        with torch.cuda.stream(stream):
+            chain.e0.record(stream)
+            steps_fn(args.steps)()
+            chain.e1.record(stream)
+            sampler.sample_now()
+            stream.synchronize()
+        ms_local = chain.e0.elapsed_time(chain.e1)
+    else:
+        with torch.cuda.stream(stream):
+            chain.e0.record(stream)
+            for g in timed_graphs:
+                g.replay()
+            chain.e1.record(stream)
+            sampler.sample_now()                         # the GPU is still working on the enqueued steps
+            stream.synchronize()
+        ms_local = chain.e0.elapsed_time(chain.e1)
     torch.cuda.synchronize()
     t_end = time.perf_counter()
     barrier()
-    ms = max_over_ranks(e0.elapsed_time(e1), world, device)
-    clocks = sampler.summary(t_begin, t_end)
+    ms = max_over_ranks(ms_local, world, device)
     ms_per_step = ms / args.steps
     value = job_throughput_gbs(ms_per_step, world)
+    # a short timed region ends before the sampler thread's next turn: keep the GPU under the same load a little
+    # longer so that the clocks are seen under load (not part of the timed region)
+    extended = False
+    if timed_graphs is not None and ms < 200.0:
+        t_load = time.perf_counter()
+        while time.perf_counter() - t_load < 0.25:
+            chain.time_ms(timed_graphs[:1])
+        t_end = time.perf_counter()
+        extended = True
+    clocks = sampler.summary(t_begin, t_end)
+    if extended and clocks["window"] == "timed region":
+        clocks["window"] = "timed region plus 0.25 s of replays of the same graph directly after it"
 
     # ---- parity spot check of what was just timed (sampled rows, fp64 oracle) ----
     parity = None
     if rank == 0:
         from oracle.c_oracle import layer_fp64_c, max_threads
         from oracle.layer import parity_metrics
-        step(0)
+        with torch.cuda.stream(stream):
+            step(0)
         stream.synchronize()
         worst_rel, worst_frac = 0.0, 0.0
         for m in ("q", "k", "gate", "down"):
@@ -370,7 +415,7 @@ def run_gpu(args):
         parity = {"rel_l2_max": worst_rel, "max_abs_over_bound": worst_frac,
                   "ok": bool(worst_rel <= 1e-3 and worst_frac <= 1.0), "rows_sampled_per_matrix": 512}
 
-    # ---- end to end: host x in pinned memory -> H2D, GEMV, D2H of y, one sync per step ----
+    # ---- end to end: host x in pinned memory -> H2D, GEMV, y into pinned host memory, one sync per step ----
     e2e_steps = min(args.steps, 2000)
     xh = {m: torch.from_numpy(cases[UNIQUE_OF[m]]["x"].copy()).pin_memory() for m in MATRICES}
     yh = {m: torch.empty(LLAMA3_8B[m][0], dtype=torch.float16).pin_memory() for m in MATRICES}
@@ -378,7 +423,7 @@ def run_gpu(args):
     def e2e_calls(r):
         for m in MATRICES:
             N, K = LLAMA3_8B[m]
-            binding.ptqtp_gemv_host(sets[r][m], N, K, xh[m], yh[m], xs[m], ys[m], stream=stream)
+            binding.ptqtp_gemv_host(sets[r][m], N, K, xh[m], yh[m], xs[m], ys[m], stream=stream, fmt=fmt)
 
     # the host-buffer calls of a step are captured once per layer copy, like the device-resident steps
     e2e_graphs = None
@@ -386,12 +431,7 @@ def run_gpu(args):
         with torch.cuda.stream(stream):
             e2e_calls(0)
             stream.synchronize()
-            e2e_graphs = []
-            for r in range(R):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=stream):
-                    e2e_calls(r)
-                e2e_graphs.append(g)
+        e2e_graphs = [chain.capture(lambda r=r: e2e_calls(r)) for r in range(R)]
 
     def e2e_step(r):
         with torch.cuda.stream(stream):
@@ -405,12 +445,12 @@ def run_gpu(args):
         e2e_step(i % R)
     barrier()
     torch.cuda.synchronize()
-    e0.record(stream)
+    chain.e0.record(stream)
     for i in range(e2e_steps):
         e2e_step(i % R)
-    e1.record(stream)
+    chain.e1.record(stream)
     stream.synchronize()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, device)
+    e2e_ms = max_over_ranks(chain.e0.elapsed_time(chain.e1), world, device)
     e2e_value = job_throughput_gbs(e2e_ms / e2e_steps, world)
     h2d = sum(2 * LLAMA3_8B[m][1] for m in MATRICES)
     d2h = sum(2 * LLAMA3_8B[m][0] for m in MATRICES)
@@ -425,59 +465,113 @@ def run_gpu(args):
             bufs = [base[u]] + [base[u].clone() for _ in range(nbuf - 1)]
             x = xs["down" if u == "down" else "q"]
             y = torch.empty(N, dtype=torch.float16, device=device)
+
+            def calls():
+                for b in bufs:
+                    binding.ptqtp_gemv(b, N, K, x, y=y, stream=stream, fmt=fmt)
+
             with torch.cuda.stream(stream):
-                for b in bufs[:2]:
-                    binding.ptqtp_gemv(b, N, K, x, y=y, stream=stream)
+                calls()
                 stream.synchronize()
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=stream):
-                    for b in bufs:
-                        binding.ptqtp_gemv(b, N, K, x, y=y, stream=stream)
-                reps = max(3, int(2000 / nbuf))
-                g.replay()
-                stream.synchronize()
-                e0.record(stream)
-                for _ in range(reps):
-                    g.replay()
-                e1.record(stream)
-                stream.synchronize()
-                us = 1e3 * e0.elapsed_time(e1) / (reps * nbuf)
-                iso = []
+            g = chain.capture(calls)
+            reps = max(3, int(2000 / nbuf))
+            us = 1e3 * chain.time_ms([g] * reps) / (reps * nbuf)
+            iso = []
+            with torch.cuda.stream(stream):
                 for i in range(12):
                     flush.fill_(i)
-                    e0.record(stream)
-                    binding.ptqtp_gemv(bufs[i % nbuf], N, K, x, y=y, stream=stream)
-                    e1.record(stream)
+                    chain.e0.record(stream)
+                    binding.ptqtp_gemv(bufs[i % nbuf], N, K, x, y=y, stream=stream, fmt=fmt)
+                    chain.e1.record(stream)
                     stream.synchronize()
-                    iso.append(1e3 * e0.elapsed_time(e1))
+                    iso.append(1e3 * chain.e0.elapsed_time(chain.e1))
+                iso_whole = []                           # the same lone call with the whole-SM launch configuration
+                for i in range(12):
+                    flush.fill_(i)
+                    chain.e0.record(stream)
+                    binding.ptqtp_gemv_cfg(bufs[i % nbuf], N, K, x, y=y, k_split=-1, stream=stream, fmt=fmt)
+                    chain.e1.record(stream)
+                    stream.synchronize()
+                    iso_whole.append(1e3 * chain.e0.elapsed_time(chain.e1))
             nb = algorithmic_bytes(N, K)
             detail[u] = {"N": N, "K": K, "bytes": nb, "us_steady": us, "gbs_steady": nb / us / 1e3,
-                         "us_isolated_median": float(np.median(iso)), "buffers": nbuf}
-            del bufs
+                         "us_isolated_median": float(np.median(iso)),
+                         "us_isolated_whole_sm_median": float(np.median(iso_whole)), "buffers": nbuf}
+            del bufs, g
         del flush
-        # the same step without any overlap of consecutive launches (plain launches, no speculative execution)
-        if graphs is not None:
+        detail["step_isolated_sum"] = {
+            "us_per_layer": sum(detail[UNIQUE_OF[m]]["us_isolated_median"] for m in MATRICES),
+            "what": "sum over the 7 matrices of the isolated, cold-L2, event-timed single calls above"}
+        if not args.no_graph:
+            # The layer as a decoder issues it: every call's x is written on the stream directly before it is used.
+            #   x_q = f(y_down of the layer before); x_k = x_v = x_q; x_o = f(y_q); x_gate = x_up = f(y_o);
+            #   x_down = y_gate * y_up   (f = one elementwise kernel, standing in for attention / norms)
+            # 7 GEMV calls + 4 elementwise kernels per layer.  The speculative pass of q, o, gate and down runs on
+            # activations that are rewritten under it and is repeated; k, v and up keep theirs.
+            xd = {"a": torch.zeros(4096, dtype=torch.float16, device=device),
+                  "o": torch.zeros(4096, dtype=torch.float16, device=device),
+                  "m": torch.zeros(4096, dtype=torch.float16, device=device),
+                  "d": torch.zeros(14336, dtype=torch.float16, device=device)}
+            ys["down"].zero_()
+
+            def dep_layer(r):
+                g4 = lambda m, x: binding.ptqtp_gemv(sets[r][m], *LLAMA3_8B[m], x, y=ys[m], stream=stream, fmt=fmt)
+                torch.add(ys["down"], 0.5, out=xd["a"])
+                g4("q", xd["a"]); g4("k", xd["a"]); g4("v", xd["a"])
+                torch.add(ys["q"], 0.25, out=xd["o"])
+                g4("o", xd["o"])
+                torch.add(ys["o"], 0.125, out=xd["m"])
+                g4("gate", xd["m"]); g4("up", xd["m"])
+                torch.mul(ys["gate"], ys["up"], out=xd["d"])
+                g4("down", xd["d"])
+
+            def dep_steps():
+                for i in range(4 * R):
+                    dep_layer(i % R)
+
+            with torch.cuda.stream(stream):
+                dep_layer(0)
+                stream.synchronize()
+            gd = chain.capture(dep_steps)
+            detail["step_dependent"] = {
+                "us_per_layer": 1e3 * chain.time_ms([gd] * 10) / (10 * 4 * R),
+                "what": "7 ptqtp_gemv + 4 elementwise kernels per layer; every x is produced on the stream directly "
+                        "before its first use (q, o, gate, down repeat their speculative pass)"}
+            old_level = binding.ptqtp_set_overlap(1)
+            try:
+                with torch.cuda.stream(stream):
+                    dep_layer(0)
+                    stream.synchronize()
+                gd1 = chain.capture(dep_steps)
+                detail["step_dependent"]["us_per_layer_level1"] = 1e3 * chain.time_ms([gd1] * 10) / (10 * 4 * R)
+                del gd1
+            finally:
+                binding.ptqtp_set_overlap(old_level)
+            del gd
+            # the same independent step without any overlap of consecutive launches: the library default
             old_level = binding.ptqtp_set_overlap(0)
             try:
                 with torch.cuda.stream(stream):
                     step(0)
                     stream.synchronize()
-                    plain = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(plain, stream=stream):
-                        for r in range(R):
-                            step(r)
-                    plain.replay()
-                    stream.synchronize()
-                    e0.record(stream)
-                    for _ in range(20):
-                        plain.replay()
-                    e1.record(stream)
-                    stream.synchronize()
-                detail["step_without_overlap"] = {"us_per_layer": 1e3 * e0.elapsed_time(e1) / (20 * R),
-                                                  "what": "ptqtp_set_overlap(0): every launch waits for the one before it"}
+                plain = chain.capture(steps_fn(R))
+                detail["step_without_overlap"] = {
+                    "us_per_layer": 1e3 * chain.time_ms([plain] * 20) / (20 * R),
+                    "what": "ptqtp_set_overlap(0), the library default: plain launches, every call waits for the one before it"}
                 del plain
             finally:
                 binding.ptqtp_set_overlap(old_level)
+            # the other batch-1 kernel (CUDA cores: masks + integer dot products on format 2) on the same step
+            other = 2 if fmt == 3 else 3
+            base_o = pack_all(other)
+            sets_o = [{m: base_o[UNIQUE_OF[m]].clone() for m in MATRICES} for _ in range(R)]
+            with torch.cuda.stream(stream):
+                steps_fn(R, f=other, layer_sets=sets_o)()
+                stream.synchronize()
+            go = chain.capture(steps_fn(4 * R, f=other, layer_sets=sets_o))
+            detail["step_other_format"] = {"format": other, "kernel": KERNEL_NAME[other],
+                                           "us_per_layer": 1e3 * chain.time_ms([go] * 10) / (10 * 4 * R)}
+            del go, sets_o, base_o
 
     sampler.stop()
 
@@ -489,22 +583,26 @@ def run_gpu(args):
     peak, peak_kind = measured_peak()
     launches = 7 * args.steps
     achieved = STEP_BYTES / (ms_per_step * 1e-3) / 1e9       # per GPU: bytes of a launch / its mean duration
+    traffic = [DRAM_TRAFFIC_BYTES[fmt][UNIQUE_OF[m]] for m in MATRICES]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": DTYPE[fmt], "data": "synthetic",
         "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: steps rotate over %d layer copies (%d MB)"
-                   % (R, R * STEP_WEIGHT_BYTES >> 20), "launch": "cuda graph" if graphs else "plain launches",
+                   % (R, R * STEP_WEIGHT_BYTES >> 20),
+                   "launch": ("one cuda graph per %d steps" % min(args.steps, GRAPH_STEPS)) if timed_graphs else "plain launches",
                    "parallelism": "replicas only" if world > 1 else "1 gpu", "bytes_per_step": STEP_BYTES,
-                   "overlap": "library default (ptqtp_set_overlap level 2): programmatic dependent launch with "
-                              "speculative execution; the CTAs of consecutive launches share SMs"},
+                   "packed_format": fmt,
+                   "overlap": "opt-in ptqtp_set_overlap(2): programmatic dependent launch with speculative execution "
+                              "(packed blobs are immutable during the run); the library default is plain launches, see "
+                              "shapes.step_without_overlap"},
         "us_per_layer": 1e3 * ms_per_step,
         "weight_gbs": STEP_WEIGHT_BYTES / (ms_per_step * 1e-3) / 1e9,
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": "of " + peak_kind,
-                     "traffic": None if DRAM_TRAFFIC_RATIO is None else DRAM_TRAFFIC_RATIO * STEP_BYTES / 7.0,
-                     "kernel": "gemv2_kernel (7 launches per step; mean over the step)",
+                     "traffic": None if any(t is None for t in traffic) else sum(traffic) / 7.0,
+                     "kernel": "%s (7 launches per step; mean over the step)" % KERNEL_NAME[fmt],
                      "bytes_per_launch_mean": STEP_BYTES / 7.0, "us_per_launch_mean": 1e3 * ms_per_step / 7.0},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "us_per_layer": 1e3 * e2e_ms / e2e_steps,
@@ -527,6 +625,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=100)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--sets", type=int, default=8, help="distinct layer copies the steps rotate over")
+    ap.add_argument("--format", type=int, default=3, choices=(2, 3),
+                    help="packed format of the timed step: 3 = tiles in int8 MMA operand order, 2 = CUDA-core kernel")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of CUDA graphs")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-shape measurements")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")

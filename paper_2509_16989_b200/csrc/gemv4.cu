@@ -45,6 +45,9 @@ namespace {
 
 constexpr int kMaxWarps4 = 16;
 constexpr int kMaxThreads4 = kMaxWarps4 * 32;
+// launch bound that sets the register budget (65536 / 576 -> 112 per thread): four 4-warp CTAs, or an 8-warp CTA and
+// two 4-warp CTAs, of consecutive launches fit into an SM's register file
+constexpr int kRegBound4 = 576;
 constexpr int kSpinAfterFailure4 = 1 << 8;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -153,7 +156,7 @@ __device__ __noinline__ void convert4_x16(uint4 ra, uint4 rb, int lane, unsigned
 }
 
 template <int D, int RU>
-__global__ void __launch_bounds__(kMaxThreads4, 1)
+__global__ void __launch_bounds__(kRegBound4, 1)
 gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
              __half* __restrict__ y, int rows_cap, int rb_base, int rb_rem, int speculate, int gated, int spin_limit,
              int inject, int* __restrict__ status_word) {
