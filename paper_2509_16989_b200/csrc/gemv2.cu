@@ -413,21 +413,8 @@ template <int D, int RU>
 ptqtp_status launch_d(const Layout2& L, const void* packed, const uint16_t* x, uint16_t* y, int grid, int warps,
                       int rows_cap, size_t smem, int speculate, int gated, cudaStream_t st) {
     auto kern = gemv2_kernel<D, RU>;
-    static thread_local size_t configured[64] = {};       // per device: largest dynamic smem already allowed
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
-    if (configured[dev] == 0) {
-        // every launch asks for the largest shared-memory carveout: consecutive launches with different
-        // carveouts cannot share an SM (it drains to be reconfigured), and these kernels make no use of L1
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
-        configured[dev] = 1;
-    }
-    if (smem > 48 * 1024 && smem > configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
-        configured[dev] = smem;
-    }
+    const ptqtp_status cs = configure_once<gemv2_kernel<D, RU>>();
+    if (cs != PTQTP_OK) return cs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(warps * 32);

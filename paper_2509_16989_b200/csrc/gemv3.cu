@@ -448,21 +448,8 @@ ptqtp_status launch_gemv3(const Layout2& L, const void* packed, int m, const uin
     if (smem > budget) return !auto_depth && depth > 2 ? PTQTP_ERR_CONFIG : PTQTP_ERR_SHAPE;
     int* status_word = nullptr;                           // shared with the batch-1 CUDA-core kernel (ptqtp_kernel_status)
     if (gemv_status_word(&status_word) != PTQTP_OK) return PTQTP_ERR_CUDA;
-    static thread_local size_t configured[64] = {};       // per device: largest dynamic smem already allowed
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
-    if (configured[dev] == 0) {
-        // every launch asks for the largest shared-memory carveout: consecutive launches with different
-        // carveouts cannot share an SM (it drains to be reconfigured), and these kernels make no use of L1
-        cudaError_t e = cudaFuncSetAttribute(gemv3_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
-        configured[dev] = 1;
-    }
-    if (smem > 48 * 1024 && smem > configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(gemv3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
-        configured[dev] = smem;
-    }
+    const ptqtp_status cs = configure_once<gemv3_kernel>();
+    if (cs != PTQTP_OK) return cs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(teams * kTeamWarps * 32);

@@ -36,7 +36,6 @@
 //     computed into shared memory, then the kernel waits for earlier work of the stream, reads x again and
 //     compares bit by bit; y is written only then, and the pass is repeated if x had changed.
 #include <cuda_fp16.h>
-#include <mutex>
 #include "ptqtp_internal.h"
 
 namespace ptqtp {
@@ -402,25 +401,6 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
     }
     const int rows = min(16 * n_cta, L.n - 16 * rb0);
     for (int r = threadIdx.x; r < rows; r += cthreads) y[16 * rb0 + r] = yout[r];
-}
-
-// Once per kernel and device, process-wide: the largest shared-memory carveout (consecutive launches with
-// different carveouts cannot share an SM, and these kernels make no use of L1) and the opt-in maximum of
-// dynamic shared memory.  Both attributes belong to the process, so they are set under a lock and never lowered.
-template <auto Kern>
-ptqtp_status configure_once() {
-    static std::mutex mu;
-    static bool done[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PTQTP_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(mu);
-    if (!done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(Kern, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
-        done[dev] = true;
-    }
-    return PTQTP_OK;
 }
 
 template <int D, int RU>

@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libptqtp (not part of the ABI).
 #pragma once
 #include <cuda_runtime.h>
+#include <mutex>
 #include <stdint.h>
 #include <stddef.h>
 #include "ptqtp.h"
@@ -157,5 +158,27 @@ bool overlap_enabled();           // programmatic dependent launch of the GEMV k
 int wait_poll_limit();            // polls of an mbarrier before a bounded wait gives up (ptqtp_set_wait_limit)
 bool take_injected_wait_failure();   // test hook: true once per armed failure (ptqtp_test_fail_next_wait)
 bool consume_pack(cudaStream_t st);   // true once after ptqtp_pack on this stream: the next GEMV launch is plain
+
+// Once per kernel and device, process-wide: the largest shared-memory carveout (consecutive launches with
+// different carveouts cannot share an SM, and these kernels make no use of L1) and the opt-in maximum of
+// dynamic shared memory.  Both attributes belong to the process, so they are set under a lock and never lowered.
+// with_carveout = false leaves the carveout preference alone (kernels that want L1).
+template <auto Kern>
+inline ptqtp_status configure_once(bool with_carveout = true) {
+    static std::mutex mu;
+    static bool done[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PTQTP_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!done[dev]) {
+        cudaError_t e = with_carveout ? cudaFuncSetAttribute(Kern, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared)
+                                      : cudaSuccess;
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
+        done[dev] = true;
+    }
+    return PTQTP_OK;
+}
+
 
 }  // namespace ptqtp

@@ -321,14 +321,8 @@ ptqtp_status launch3(const Layout2& L, const void* packed, const unsigned char* 
     auto kern = skinny3_kernel<NTT>;
     const int depth = smem3(NTT, warps, 3) <= 227 * 1024 ? 3 : 2;         // ring slots per compute warp
     const size_t smem = smem3(NTT, warps, depth);
-    static thread_local size_t configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
-    if (smem > 48 * 1024 && smem > configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) { set_last_cuda_error(e); return PTQTP_ERR_CUDA; }
-        configured[dev] = smem;
-    }
+    const ptqtp_status cs = configure_once<skinny3_kernel<NTT>>(false);
+    if (cs != PTQTP_OK) return cs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3((warps + 1) * 32);                               // + the tile loader warp

@@ -1,6 +1,10 @@
 """Measurements of the workloads other than the benchmark's headline step (run on a B200).
 
-    python -m paper_2509_16989_b200.report [--only 0,2,3]
+    python -m paper_2509_16989_b200.report [--only 0,2,3] [--format 3]
+
+Batch-1 calls use the packed format given by --format (default 3: tiles in int8 MMA operand order; 2: the
+CUDA-core kernel); the small-batch calls (M > 1) always use format 2.  The program opts in to overlap level 2, as
+a decoder would whose packed blobs never change while GEMV calls are in flight.
 
   0  Qwen3-0.6B up_proj 3072 x 1024, batch 1
   2  batch sweep M in {1,...,64} of ptqtp_gemm_skinny on the 14336 x 4096 gate/up shape (and ptqtp_gemv at M = 1)
@@ -10,8 +14,9 @@
      slice y): five or four calls per layer instead of seven
   6  the seven linears of a LLaMA-3-70B-shaped layer as one chain of calls
 
-(The 32-layer stack built from decomposed weights needs the CPU oracle to prepare its inputs and is therefore
-measured by tests/test_gpu_stack.py.)
+(The 32-layer stack built from decomposed weights needs planes from the decomposition of Algorithm 1, which this
+package does not contain; tests/test_gpu_stack.py builds it with the CPU oracle and checks parity on it.  Its
+timing per layer is that of the benchmark's step: the kernels are branch-free in the plane values.)
 
 Every timing is a CUDA-event steady state inside a CUDA graph that walks over distinct packed buffers
 totalling more than twice the L2 size, so the planes come from HBM.  One JSON line per result.
@@ -30,6 +35,8 @@ if ROOT not in sys.path:
 
 from paper_2509_16989_b200 import binding  # noqa: E402
 from paper_2509_16989_b200.inputs import LLAMA3_8B, LLAMA3_70B, QWEN3_0P6B_UP, make_case  # noqa: E402
+
+FMT = binding.FORMAT_V3          # packed format of the batch-1 calls (--format)
 
 
 def algorithmic_bytes(N, K, M=1):
@@ -79,15 +86,21 @@ def emit(**kw):
 
 def gemv_case(T, name, N, K, p_zero=0.4, seed=0, batches=(1,)):
     c = make_case(N, K, seed=seed, M=max(batches), p_zero=p_zero)
-    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
-    bufs = T.copies(packed)
     Xall = dev(np.atleast_2d(c["x"]))
+    packed, bufs = None, None
     for M in batches:
+        want = FMT if M == 1 else binding.FORMAT_V2
+        if packed is None or want != have:
+            del packed, bufs
+            torch.cuda.empty_cache()
+            packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=want)
+            bufs = T.copies(packed)
+            have = want
         if M == 1:
             x = Xall[0].contiguous()
             y = torch.empty(N, dtype=torch.float16, device="cuda")
-            us = T.steady_us([lambda b=b: binding.ptqtp_gemv(b, N, K, x, y=y, stream=T.stream) for b in bufs])
-            call = "ptqtp_gemv"
+            us = T.steady_us([lambda b=b: binding.ptqtp_gemv(b, N, K, x, y=y, stream=T.stream, fmt=FMT) for b in bufs])
+            call = "ptqtp_gemv (format %d)" % FMT
         else:
             X = Xall[:M].contiguous()
             Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
@@ -113,7 +126,7 @@ def config0(T):
 def config2(T):
     N, K = LLAMA3_8B["gate"]
     c = make_case(N, K, seed=2, M=64)
-    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
+    packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=binding.FORMAT_V2)
     bufs = T.copies(packed)
     Xall = dev(c["x"])
     for M in (1, 2, 4, 8, 16, 32, 64):
@@ -150,7 +163,7 @@ def config5(T):
         base = {}
         for i, (name, N, K) in enumerate(shapes):
             c = make_case(N, K, seed=50 + i)
-            packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
+            packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=FMT)
             base[name] = (packed, dev(c["x"]), torch.empty(N, dtype=torch.float16, device="cuda"))
         layer_bytes = sum(base[n][0].numel() for n, _, _ in shapes)
         copies = max(4, -(-(2 * T.l2 + (64 << 20)) // layer_bytes))
@@ -160,13 +173,13 @@ def config5(T):
             for name, N, K in shapes:
                 if name == "swiglu":
                     calls.append(lambda p=layers[l][name], N=N, K=K, x=base[name][1], y=base[name][2][:N // 2]:
-                                 binding.ptqtp_gemv_swiglu(p, N, K, x, y=y, stream=T.stream))
+                                 binding.ptqtp_gemv_swiglu(p, N, K, x, y=y, stream=T.stream, fmt=FMT))
                 else:
                     calls.append(lambda p=layers[l][name], N=N, K=K, x=base[name][1], y=base[name][2]:
-                                 binding.ptqtp_gemv(p, N, K, x, y=y, stream=T.stream))
+                                 binding.ptqtp_gemv(p, N, K, x, y=y, stream=T.stream, fmt=FMT))
         us = T.steady_us(calls) * len(shapes)
         nb = sum(algorithmic_bytes(N, K) - (N if name == "swiglu" else 0) for name, N, K in shapes)
-        emit(workload="cfg5 llama3-8b layer, " + what, call="%d x ptqtp_gemv" % len(shapes), us_per_layer=round(us, 3),
+        emit(workload="cfg5 llama3-8b layer, " + what, call="%d x ptqtp_gemv (format %d)" % (len(shapes), FMT), us_per_layer=round(us, 3),
              gbs=round(nb / us / 1e3, 1), bytes=nb, layer_copies=copies)
         del layers, base, calls
         torch.cuda.empty_cache()
@@ -179,27 +192,31 @@ def config6(T):
     for i, u in enumerate(sorted(LLAMA3_70B)):
         N, K = LLAMA3_70B[u]
         c = make_case(N, K, seed=60 + i)
-        packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]))
+        packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=FMT)
         base[u] = (packed, dev(c["x"]), torch.empty(N, dtype=torch.float16, device="cuda"))
     calls = []
     for l in range(2):
         for name, u in order:
             p = base[u][0] if (l == 0 and name in ("q", "k", "gate", "down")) else base[u][0].clone()
             N, K = LLAMA3_70B[u]
-            calls.append(lambda p=p, N=N, K=K, x=base[u][1], y=base[u][2]: binding.ptqtp_gemv(p, N, K, x, y=y, stream=T.stream))
+            calls.append(lambda p=p, N=N, K=K, x=base[u][1], y=base[u][2]: binding.ptqtp_gemv(p, N, K, x, y=y, stream=T.stream, fmt=FMT))
     us = T.steady_us(calls, reps=40) * len(order)
     nb = sum(algorithmic_bytes(*LLAMA3_70B[u]) for _, u in order)
-    emit(workload="cfg6 llama3-70b-shaped layer as one chain", call="7 x ptqtp_gemv", us_per_layer=round(us, 3),
+    emit(workload="cfg6 llama3-70b-shaped layer as one chain", call="7 x ptqtp_gemv (format %d)" % FMT, us_per_layer=round(us, 3),
          gbs=round(nb / us / 1e3, 1), bytes=nb, layer_copies=2)
 
 
 def main():
+    global FMT
     ap = argparse.ArgumentParser()
     ap.add_argument("--only", default="0,2,3,5,6")
+    ap.add_argument("--format", type=int, default=3, choices=(2, 3))
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise RuntimeError("needs a CUDA device")
     binding.lib()
+    FMT = args.format
+    binding.ptqtp_set_overlap(2)
     T = Timer()
     which = set(int(v) for v in args.only.split(","))
     if 0 in which:
@@ -212,6 +229,7 @@ def main():
         config5(T)
     if 6 in which:
         config6(T)
+
 
 
 if __name__ == "__main__":
