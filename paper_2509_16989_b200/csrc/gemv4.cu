@@ -157,8 +157,8 @@ __device__ __noinline__ void convert4_x16(uint4 ra, uint4 rb, int lane, unsigned
 template <int D, int RU>
 __global__ void __launch_bounds__(kRegBound4, 1)
 gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
-             __half* __restrict__ y, int rows_cap, int rb_base, int rb_rem, int speculate, int gated, int spin_limit,
-             int inject, int* __restrict__ status_word) {
+             __half* __restrict__ y, int rows_cap, int rb_base, int rb_rem, int speculate, int overlap, int gated,
+             int spin_limit, int inject, int* __restrict__ status_word) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int S = L.sbs;
     const int warps = blockDim.x >> 5;
@@ -242,22 +242,31 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
     for (int attempt = 0; attempt < 2; ++attempt) {
         // Pass 0 is speculative when allowed: x is read before earlier work of the stream is known to be complete.
         const bool spec = speculate && attempt == 0;
-        // The packed planes do not depend on earlier work of the stream: the ring is filled before any wait.
+        // x as it is, by one bulk copy (through L2, the point of coherence): one round trip whatever K is.  It is
+        // requested before the ring is filled (copies complete in the order they were requested: behind a full
+        // ring x would arrive microseconds later), except under a dependent launch without speculative execution,
+        // where the planes, which do not depend on earlier work of the stream, are requested before the wait.
         pt = n_rb > 0 ? 0 : n_sl;
         pleft = n_rb;
         psrc = codes + tile_offset3(L, rbw, min(sl_lane, S - 1));
+        const bool fill_first = !spec && !waited && overlap;
+        if (fill_first) {
 #pragma unroll
-        for (int d = 0; d < D; ++d) issue();
+            for (int d = 0; d < D; ++d) issue();
+        }
         if (!spec && !waited) {
             asm volatile("griddepcontrol.wait;" ::: "memory");
             waited = true;
         }
-        // x as it is, by one bulk copy (through L2, the point of coherence): one round trip whatever K is
         if (threadIdx.x == 0) {
             mbar_expect_tx(xbar_a, xbytes);
             bulk_copy_g2s(smem_u32(raw), x, xbytes, xbar_a);
         }
         __syncthreads();                                // the mbarrier of x is initialised and armed before anyone polls it
+        if (!fill_first) {                              // (and x has been requested before any tile)
+#pragma unroll
+            for (int d = 0; d < D; ++d) issue();
+        }
         if (!mbar_try_wait(xbar_a, (uint32_t)attempt)) {
             const int limit = failed ? kSpinAfterFailure4 : spin_limit;
             int spins = 0;
@@ -422,7 +431,7 @@ ptqtp_status launch_d4(const Layout3& L, const void* packed, const uint16_t* x, 
     cfg.numAttrs = overlap_enabled() && !consume_pack(st) ? 1 : 0;   // plain right after a pack on this stream
     cudaError_t e = cudaLaunchKernelEx(&cfg, gemv4_kernel<D, RU>, L, static_cast<const unsigned char*>(packed),
                                        reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap,
-                                       L.nrb / grid, L.nrb % grid, speculate, gated, wait_poll_limit(),
+                                       L.nrb / grid, L.nrb % grid, speculate, overlap_enabled() ? 1 : 0, gated, wait_poll_limit(),
                                        take_injected_wait_failure() ? 1 : 0, status_word);
     if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
     return PTQTP_OK;
