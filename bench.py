@@ -548,6 +548,39 @@ def run_gpu(args):
             finally:
                 binding.ptqtp_set_overlap(old_level)
             del gd
+            # Four launches per layer (format 3): q, k, v in one launch and gate, up with the gated pair epilogue in
+            # one launch (ptqtp_gemv_multi over the separately packed blobs), o and down as before.  First with
+            # independent activations like the headline step, then as a decoder issues it: down reads the gated
+            # output directly, the other activations come from one elementwise kernel each.
+            if fmt == 3:
+                yg = torch.zeros(14336, dtype=torch.float16, device=device)
+
+                def four(r, dep):
+                    S_ = sets[r]
+                    if dep:
+                        torch.add(ys["down"], 0.5, out=xd["a"])
+                    binding.ptqtp_gemv_multi([S_["q"], S_["k"], S_["v"]], [4096, 1024, 1024], 4096, xd["a"] if dep else xs["q"],
+                                             ys=[ys["q"], ys["k"], ys["v"]], stream=stream)
+                    if dep:
+                        torch.add(ys["q"], 0.25, out=xd["o"])
+                    binding.ptqtp_gemv(S_["o"], 4096, 4096, xd["o"] if dep else xs["o"], y=ys["o"], stream=stream, fmt=3)
+                    if dep:
+                        torch.add(ys["o"], 0.125, out=xd["m"])
+                    binding.ptqtp_gemv_multi([S_["gate"], S_["up"]], [14336, 14336], 4096, xd["m"] if dep else xs["gate"],
+                                             ys=[yg], epilogue=binding.EPILOGUE_GATED_PAIR, stream=stream)
+                    binding.ptqtp_gemv(S_["down"], 4096, 14336, yg if dep else xs["down"], y=ys["down"], stream=stream, fmt=3)
+
+                four_bytes = STEP_BYTES - 2 * 2 * 4096 - 2 * 4096 - 2 * 14336      # x of k, v, up and one y not moved
+                for dep, key in ((False, "four_launch_layer"), (True, "four_launch_layer_dependent")):
+                    with torch.cuda.stream(stream):
+                        four(0, dep)
+                        stream.synchronize()
+                    g4l = chain.capture(lambda dep=dep: [four(i % R, dep) for i in range(4 * R)])
+                    us4 = 1e3 * chain.time_ms([g4l] * 10) / (10 * 4 * R)
+                    detail[key] = {"us_per_layer": us4, "gbs": four_bytes / us4 / 1e3, "bytes": four_bytes,
+                                   "launches": "ptqtp_gemv_multi(q,k,v) + ptqtp_gemv(o) + ptqtp_gemv_multi(gate,up; gated pair) "
+                                               "+ ptqtp_gemv(down)" + (" + 3 elementwise kernels; down reads the gated output" if dep else "")}
+                    del g4l
             # the same independent step without any overlap of consecutive launches: the library default
             old_level = binding.ptqtp_set_overlap(0)
             try:

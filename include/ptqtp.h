@@ -170,6 +170,23 @@ PTQTP_API ptqtp_status ptqtp_gemv(const ptqtp_shape *shape /* host */, const voi
 PTQTP_API ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                                const uint16_t *x, uint16_t *y, void *stream);
 
+/* Several matrices that share their input in ONE launch: y[j] = layer_j(x) for j < count, 1 <= count <= 4 -- the
+ * q, k and v projections of an attention block, or the gate and up projections of an MLP (Eq. 1-2 per matrix; the
+ * paper reports decode speed for the model as a whole, Sec. 4 "End-to-End Speed", where these share x).  The blobs
+ * are packed separately (format 3 each, PTQTP_ERR_CONFIG otherwise) and need only agree in K (PTQTP_ERR_SHAPE
+ * otherwise).  shapes, packed, packed_bytes, y: host arrays of `count` entries; packed[j], x, y[j]: device.
+ * x is fetched, converted and (under overlap level 2) verified once; every y[j] holds exactly the bits that
+ * ptqtp_gemv gives for that matrix alone.
+ * epilogue: PTQTP_EPILOGUE_NONE, or PTQTP_EPILOGUE_GATED_PAIR for count == 2 and equal N: matrix 0 is the gate,
+ * matrix 1 the up projection, and ONE output y[0][i] = silu(t0[i]) * t1[i] (t = the fp32 row sums before any
+ * rounding, silu(g) = g / (1 + exp(-g))) is written, rounded once to fp16; y[1] is ignored and may be NULL. */
+#define PTQTP_EPILOGUE_NONE 0
+#define PTQTP_EPILOGUE_GATED_PAIR 1
+PTQTP_API ptqtp_status ptqtp_gemv_multi(int32_t count, const ptqtp_shape *shapes /* host */,
+                              const void *const *packed /* host array */, const size_t *packed_bytes /* host */,
+                              const uint16_t *x, uint16_t *const *y /* host array */, int32_t epilogue,
+                              void *stream);
+
 /* Small-batch variant: Y[m,:] = layer(X[m,:]) for m < M, 1 <= M <= PTQTP_MAX_BATCH.
  * X: device fp16 [M*K] row-major; Y: device fp16 [M*N] row-major.  Same definition per row of X.
  * Format 2, M >= 2: the planes are contracted on the tensor cores with int8 warp MMAs against 15-bit

@@ -26,7 +26,7 @@ EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptq
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
            "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws",
            "ptqtp_gemm_skinny_static", "ptqtp_kernel_status", "ptqtp_gemv_swiglu", "ptqtp_kernel_status_clear",
-           "ptqtp_set_wait_limit", "ptqtp_test_fail_next_wait")
+           "ptqtp_set_wait_limit", "ptqtp_test_fail_next_wait", "ptqtp_gemv_multi")
 
 
 class PtqtpError(RuntimeError):
@@ -64,6 +64,8 @@ def lib():
         L.ptqtp_gemv.argtypes = [sp, vp, sz, vp, vp, vp]
         L.ptqtp_gemv_swiglu.restype = ctypes.c_int
         L.ptqtp_gemv_swiglu.argtypes = [sp, vp, sz, vp, vp, vp]
+        L.ptqtp_gemv_multi.restype = ctypes.c_int
+        L.ptqtp_gemv_multi.argtypes = [i32, sp, ctypes.POINTER(vp), ctypes.POINTER(sz), vp, ctypes.POINTER(vp), i32, vp]
         L.ptqtp_gemm_skinny.restype = ctypes.c_int
         L.ptqtp_gemm_skinny.argtypes = [sp, vp, sz, i32, vp, vp, vp]
         L.ptqtp_gemm_skinny_workspace_size.restype = sz
@@ -197,6 +199,26 @@ def ptqtp_gemv_swiglu(packed, N, K, x, y=None, stream=None, fmt=FORMAT_V2):
                                  _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"), _stream_ptr(stream))
     _check(st, "ptqtp_gemv_swiglu")
     return y
+
+
+EPILOGUE_NONE, EPILOGUE_GATED_PAIR = 0, 1
+
+
+def ptqtp_gemv_multi(packed_list, N_list, K, x, ys=None, epilogue=EPILOGUE_NONE, stream=None):
+    """One launch for several format-3 matrices that share x: returns the list of outputs (one output for the
+    gated pair epilogue: silu(matrix 0) * matrix 1)."""
+    count = len(packed_list)
+    shapes = (Shape * count)(*[make_shape(N, K, fmt=FORMAT_V3) for N in N_list])
+    n_out = 1 if epilogue == EPILOGUE_GATED_PAIR else count
+    if ys is None:
+        ys = [torch.empty(N_list[j], dtype=torch.float16, device=x.device) for j in range(n_out)]
+    ptrs = (ctypes.c_void_p * count)(*[_dev(p, torch.uint8, "packed").value for p in packed_list])
+    sizes = (ctypes.c_size_t * count)(*[p.numel() for p in packed_list])
+    yp = (ctypes.c_void_p * count)(*([_dev(y, torch.float16, "y").value for y in ys] + [None] * (count - len(ys))))
+    st = lib().ptqtp_gemv_multi(count, shapes, ptrs, sizes, _dev(x, torch.float16, "x"), yp, int(epilogue),
+                                _stream_ptr(stream))
+    _check(st, "ptqtp_gemv_multi")
+    return ys
 
 
 def ptqtp_gemm_skinny(packed, N, K, X, Y=None, stream=None, fmt=None):

@@ -191,6 +191,30 @@ ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape* shape, const void* packed, siz
     return launch_gemv2(L.l2, packed, x, y, 0, 0, 0, 0, static_cast<cudaStream_t>(stream), true);
 }
 
+ptqtp_status ptqtp_gemv_multi(int32_t count, const ptqtp_shape* shapes, const void* const* packed,
+                              const size_t* packed_bytes, const uint16_t* x, uint16_t* const* y, int32_t epilogue,
+                              void* stream) {
+    if (!shapes || !packed || !packed_bytes || !x || !y) return PTQTP_ERR_NULL;
+    if (count < 1 || count > kMaxJobs4) return PTQTP_ERR_SHAPE;
+    if (epilogue != PTQTP_EPILOGUE_NONE && epilogue != PTQTP_EPILOGUE_GATED_PAIR) return PTQTP_ERR_CONFIG;
+    if (!aligned16(x)) return PTQTP_ERR_ALIGN;
+    const bool pair = epilogue == PTQTP_EPILOGUE_GATED_PAIR;
+    if (pair && (count != 2 || shapes[0].n_out != shapes[1].n_out)) return PTQTP_ERR_SHAPE;
+    Jobs4 J = {};
+    for (int j = 0; j < count; ++j) {
+        AnyLayout L;
+        ptqtp_status s = check_packed(&shapes[j], packed[j], packed_bytes[j], &L);
+        if (s != PTQTP_OK) return s;
+        if (!L.v3) return PTQTP_ERR_CONFIG;
+        if (shapes[j].k_in != shapes[0].k_in) return PTQTP_ERR_SHAPE;
+        uint16_t* yj = pair && j == 1 ? y[0] : y[j];     // the pair has one output
+        if (!yj) return PTQTP_ERR_NULL;
+        if (!aligned16(yj)) return PTQTP_ERR_ALIGN;
+        add_job4(J, L.l3, packed[j], yj);
+    }
+    return launch_gemv4_jobs(J, x, 0, 0, 0, 0, static_cast<cudaStream_t>(stream), pair ? 2 : 0);
+}
+
 ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, int32_t m,
                                const uint16_t* X, uint16_t* Y, void* stream) {
     if (!X || !Y) return PTQTP_ERR_NULL;

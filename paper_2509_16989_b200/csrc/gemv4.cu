@@ -46,7 +46,7 @@ constexpr int kMaxWarps4 = 16;
 constexpr int kMaxThreads4 = kMaxWarps4 * 32;
 // launch bound that sets the register budget (65536 / 576 -> 112 per thread): four 4-warp CTAs, or an 8-warp CTA and
 // two 4-warp CTAs, of consecutive launches fit into an SM's register file
-constexpr int kRegBound4 = 576;
+constexpr int kRegBound4 = 512;
 constexpr int kSpinAfterFailure4 = 1 << 8;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -78,7 +78,8 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
 }
 
 // Shared memory: x as read (fp16, 2 K bytes), one staging area per warp (the superblock the warp is on, in
-// B-fragment order, 1024 bytes, then its four group records: 2^-s as float bits, sum of the group's integers), the
+// B-fragment order, 1024 bytes, then its four group records: 2^-s as float bits, sum of the group's integers, then
+// the warp's share of every job: first row block, row blocks, first row among the CTA's rows), the
 // per-superblock partial sums, the output rows (fp16), the mbarriers (one per ring slot, then one for x), then
 // the ring (RU tiles per slot, D slots per warp).
 //
@@ -86,16 +87,17 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
 // which half of a k-step's 8 columns), 16 bytes at 256 q + 16 slot: the words of k-steps 4q .. 4q+3, word i
 // holding the bytes of columns 128 j + 8 i + 4 th + 0..3.  The lane with g = 2 j + hl and t = 2 (j % 2) + th
 // reads its 16 words with four 128-bit loads; the other lanes hold zeros.
-constexpr int kStage4 = 1024 + 64;
+constexpr int kStage4 = 1024 + 32 + 64;            // B-fragment words, four group records, the warp's job table
 struct Smem4 {
-    size_t stage_off, partial_off, yout_off, bar_off, ring_off, total;
+    size_t stage_off, partial_off, yout_off, jobs_off, bar_off, ring_off, total;
 };
 __host__ __device__ inline Smem4 smem_layout4(int k, int sbs, int rows_cap, int warps, int depth, int ru) {
     Smem4 m;
     m.stage_off = (size_t)2 * k;
     m.partial_off = m.stage_off + (size_t)warps * kStage4;
     m.yout_off = m.partial_off + (size_t)rows_cap * sbs * 4;
-    m.bar_off = (m.yout_off + (size_t)rows_cap * 2 + 7) / 8 * 8;
+    m.jobs_off = (m.yout_off + (size_t)rows_cap * 2 + 15) / 16 * 16;      // the CTA's share of every job
+    m.bar_off = m.jobs_off + kMaxJobs4 * 16;
     m.ring_off = (m.bar_off + (size_t)(warps * depth + 1) * 8 + 127) / 128 * 128;
     m.total = m.ring_off + (size_t)warps * depth * ru * kTile3;
     return m;
@@ -154,15 +156,34 @@ __device__ __noinline__ void convert4_x16(uint4 ra, uint4 rb, int lane, unsigned
     if ((lane & 7) == 0) reinterpret_cast<int2*>(stage + 1024)[j] = make_int2((int)((uint32_t)(127 - s) << 23), isum);
 }
 
-template <int D, int RU>
+// This CTA's and this warp's share of job j: the CTA's row blocks [rb0, rb0 + n_cta) (balanced partition of the
+// job over the grid, the CTAs that take one block more starting at CTA rb_off[j]), of which the warp streams
+// [rbw, rbw + n_rb) (the m warps of a superblock lane split them into contiguous runs, balanced +-1).
+struct Share4 {
+    int rb0, n_cta, rbw, n_rb;
+};
+__device__ __forceinline__ Share4 share_of(const Jobs4& J, int j, int wi, int m, bool idle) {
+    int idx = (int)blockIdx.x - J.rb_off[j];
+    if (idx < 0) idx += (int)gridDim.x;
+    Share4 s;
+    s.rb0 = idx * J.rb_base[j] + min(idx, J.rb_rem[j]);
+    s.n_cta = J.rb_base[j] + (idx < J.rb_rem[j] ? 1 : 0);
+    s.rbw = s.rb0 + (idle ? 0 : wi * (s.n_cta / m) + min(wi, s.n_cta % m));
+    s.n_rb = idle ? 0 : s.n_cta / m + (wi < s.n_cta % m ? 1 : 0);
+    return s;
+}
+
+// One launch serves up to kMaxJobs4 matrices ("jobs") that share x: a warp, once on a superblock, streams its
+// tiles of job 0, then of job 1, ...; x is fetched, converted and verified once for all of them.
+// kMulti = false is the same kernel for a single matrix with the job loops folded away.
+template <int D, int RU, bool kMulti>
 __global__ void __launch_bounds__(kRegBound4, 1)
-gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* __restrict__ x,
-             __half* __restrict__ y, int rows_cap, int rb_base, int rb_rem, int speculate, int overlap, int gated,
-             int spin_limit, int inject, int* __restrict__ status_word) {
+gemv4_kernel(const __grid_constant__ Jobs4 J, const __half* __restrict__ x, int rows_cap, int speculate, int overlap,
+             int gated, int spin_limit, int inject, int* __restrict__ status_word) {
     extern __shared__ __align__(128) unsigned char smem[];
-    const int S = L.sbs;
+    const int S = J.sbs;
     const int warps = blockDim.x >> 5;
-    const Smem4 sm = smem_layout4(L.k, S, rows_cap, warps, D, RU);
+    const Smem4 sm = smem_layout4(J.k, S, rows_cap, warps, D, RU);
     uint4* raw = reinterpret_cast<uint4*>(smem);                             // x as read (fp16)
     float* partial = reinterpret_cast<float*>(smem + sm.partial_off);       // [rows_cap][S]
     __half* yout = reinterpret_cast<__half*>(smem + sm.yout_off);            // [rows_cap]: the rows as they will be stored
@@ -178,22 +199,35 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
     // Let the next kernel on the stream start while this one runs.
     asm volatile("griddepcontrol.launch_dependents;");
 
-    // this CTA's row blocks (balanced partition from the host: the first rb_rem CTAs take rb_base + 1), and this
-    // warp's share of their tiles
-    const int rb0 = (int)blockIdx.x * rb_base + min((int)blockIdx.x, rb_rem);
-    const int rb1 = rb0 + rb_base + ((int)blockIdx.x < rb_rem ? 1 : 0);
     const int Wc = min(S, warps);                       // superblock lanes among the warps
     const int m = warps / Wc;                           // warps sharing a superblock lane
     const int sl_lane = warp % Wc, wi = warp / Wc;
     const bool idle = wi >= m;
     const int n_sl = idle ? 0 : (S - sl_lane + Wc - 1) / Wc;
-    // the m warps of a superblock lane split the CTA's row blocks into contiguous runs (balanced +-1)
-    const int n_cta = rb1 - rb0;
-    const int rbw = rb0 + (idle ? 0 : wi * (n_cta / m) + min(wi, n_cta % m));
-    const int n_rb = idle ? 0 : n_cta / m + (wi < n_cta % m ? 1 : 0);
-    const unsigned char* codes = packed + L.codes_off;
-    const int nchunks = L.k >> 3, cthreads = blockDim.x;
-    const uint32_t xbytes = (uint32_t)L.k * 2u;
+    const int nchunks = J.k >> 3, cthreads = blockDim.x;
+    const uint32_t xbytes = (uint32_t)J.k * 2u;
+    const int njobs = kMulti ? J.count : 1;
+    // The shares are worked out once, by lane j for job j: the warp's into its staging area (first row block, row
+    // blocks, first row among the CTA's rows), the CTA's into a table of its own (first row block, row blocks,
+    // first row); rows_total = rows of all jobs in this CTA (16 per row block).
+    int4* wtab = reinterpret_cast<int4*>(stage + 1024 + 32);
+    int4* ctab = reinterpret_cast<int4*>(smem + sm.jobs_off);
+    int rows_total = 0;
+    {
+        const Share4 mine = share_of(J, min(lane, njobs - 1), wi, m, idle);
+        int before = 0;
+        for (int j = 0; j < njobs; ++j) {
+            int idx = (int)blockIdx.x - J.rb_off[j];
+            if (idx < 0) idx += (int)gridDim.x;
+            const int rows = 16 * (J.rb_base[j] + (idx < J.rb_rem[j] ? 1 : 0));
+            if (j < lane) before += rows;
+            rows_total += rows;
+        }
+        if (lane < njobs) {
+            wtab[lane] = make_int4(mine.rbw, mine.n_rb, before + 16 * (mine.rbw - mine.rb0), 0);
+            if (warp == 0) ctab[lane] = make_int4(mine.rb0, mine.n_cta, before, 0);
+        }
+    }
 
     if (lane == 0) {
 #pragma unroll
@@ -203,12 +237,30 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
     }
     __syncwarp();
 
-    // producer (lane 0): superblock pass pt, tiles left in it, source of the next copy, ring slot
+    // producer (lane 0): superblock pass pt and job pj of the segment being requested, tiles left in it, source of
+    // the next copy, ring slot
     const uint32_t bars_a = smem_u32(bars), ring_a = smem_u32(ring), xbar_a = smem_u32(xbar);
-    int pt = 0, pleft = 0, pslot = 0;
+    int pt = 0, pj = 0, pleft = 0, pslot = 0;
     // test hook: the first copy of warp 0 of CTA 0 announces more bytes than it brings, so its wait runs out
     uint32_t surplus = (inject && blockIdx.x == 0 && warp == 0) ? 16u : 0u;
-    const unsigned char* psrc = codes;
+    const unsigned char* psrc = nullptr;
+    auto seek = [&]() {                                 // from (pt, pj) on, the next segment that has tiles
+        while (pt < n_sl) {
+            if (pj < njobs) {
+                const int4 sh = wtab[pj];
+                if (sh.y > 0) {
+                    pleft = sh.y;
+                    psrc = J.codes[pj] + ((size_t)(sl_lane + pt * Wc) * J.nrb[pj] + sh.x) * kTile3;
+                    return;
+                }
+                ++pj;
+            } else {
+                pj = 0;
+                ++pt;
+            }
+        }
+        pleft = 0;
+    };
     auto issue = [&]() {
         if (pt < n_sl) {
             const int nun = min(RU, pleft);
@@ -221,9 +273,8 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
             psrc += bytes;
             pleft -= nun;
             if (pleft == 0) {
-                ++pt;
-                pleft = n_rb;
-                psrc = codes + tile_offset3(L, rbw, min(sl_lane + pt * Wc, S - 1));
+                ++pj;
+                seek();
             }
         }
         pslot = pslot + 1 == D ? 0 : pslot + 1;
@@ -246,9 +297,9 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
         // requested before the ring is filled (copies complete in the order they were requested: behind a full
         // ring x would arrive microseconds later), except under a dependent launch without speculative execution,
         // where the planes, which do not depend on earlier work of the stream, are requested before the wait.
-        pt = n_rb > 0 ? 0 : n_sl;
-        pleft = n_rb;
-        psrc = codes + tile_offset3(L, rbw, min(sl_lane, S - 1));
+        pt = 0;
+        pj = 0;
+        seek();
         const bool fill_first = !spec && !waited && overlap;
         if (fill_first) {
 #pragma unroll
@@ -282,7 +333,7 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
             uint32_t b0[16], b1[16];
             {
                 uint4 ra = make_uint4(0u, 0u, 0u, 0u), rb = ra;
-                if (sb * kSuper3 + 16 * lane < L.k) {
+                if (sb * kSuper3 + 16 * lane < J.k) {
                     ra = raw[sb * 64 + 2 * lane];
                     rb = raw[sb * 64 + 2 * lane + 1];
                 }
@@ -303,8 +354,10 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
             const int2 mt = reinterpret_cast<const int2*>(stage + 1024)[t];
             const float cx0 = __int_as_float(mt.x), cx1 = 0.0625f * cx0;
             const int n0 = -mt.y, n1 = -(mt.y << 2), n2 = -(mt.y << 4), n3 = -(mt.y * 85);
-            float* ppart = partial + (size_t)(16 * (rbw - rb0) + 2 * g + (t & 1)) * S + sb;
-            for (int j0 = 0; j0 < n_rb; j0 += RU) {
+            for (int jb = 0; jb < njobs; ++jb) {
+            const int4 sh = wtab[jb];                   // (first row block, row blocks, first row among the CTA's rows)
+            float* ppart = partial + (size_t)(sh.z + 2 * g + (t & 1)) * S + sb;
+            for (int j0 = 0; j0 < sh.y; j0 += RU) {
                 // wait (bounded) for the copy in slot cslot; it has normally arrived long ago
                 if (!mbar_try_wait(bars_a + 8 * cslot, phase)) {
                     const int limit = failed ? kSpinAfterFailure4 : spin_limit;
@@ -313,7 +366,7 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
                         if (++spins >= limit) { failed = true; break; }
                     }
                 }
-                const int nun = min(RU, n_rb - j0);
+                const int nun = min(RU, sh.y - j0);
                 const unsigned char* buf = ring + cslot * kSlot + lane * 16;
                 auto tile_body = [&](const unsigned char* tb, float* pp) {
                     // chains A: rows (field 0 | field 1), B: rows (field 2 | all fields); even and odd k-steps apart
@@ -350,14 +403,15 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
                 issue();
                 if (++cslot == D) { cslot = 0; phase ^= 1u; }
             }
+            }
         }
         // All partial sums of this pass are in shared memory: sum them over the superblocks in a fixed order and
         // round once to fp16 now, so that after the dependency wait only the verification of x and the store remain.
         __syncthreads();
-        if (gated) {
+        if (gated == 1) {
             // gated pair epilogue: a row pair is (gate row, up row) and gives one output silu(gate) * up, computed
             // from the unrounded fp32 sums
-            for (int r = threadIdx.x; r < 8 * n_cta; r += cthreads) {
+            for (int r = threadIdx.x; r < rows_total / 2; r += cthreads) {
                 float gt = 0.f, up = 0.f;
                 for (int s = 0; s < S; ++s) {
                     gt += partial[(size_t)(2 * r) * S + s];
@@ -365,8 +419,19 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
                 }
                 yout[r] = __float2half_rn(gt / (1.f + expf(-gt)) * up);
             }
+        } else if (gated == 2) {
+            // the same with the gate rows in job 0 and the up rows in job 1 (equal shapes, equal partitions)
+            const int half_rows = rows_total / 2;
+            for (int r = threadIdx.x; r < half_rows; r += cthreads) {
+                float gt = 0.f, up = 0.f;
+                for (int s = 0; s < S; ++s) {
+                    gt += partial[(size_t)r * S + s];
+                    up += partial[(size_t)(half_rows + r) * S + s];
+                }
+                yout[r] = __float2half_rn(gt / (1.f + expf(-gt)) * up);
+            }
         } else {
-            for (int r = threadIdx.x; r < 16 * n_cta; r += cthreads) {
+            for (int r = threadIdx.x; r < rows_total; r += cthreads) {
                 float acc = 0.f;
                 for (int s = 0; s < S; ++s) acc += partial[(size_t)r * S + s];
                 yout[r] = __float2half_rn(acc);
@@ -403,19 +468,28 @@ gemv4_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
     __syncthreads();
-    if (gated) {
-        const int npairs = min(8 * n_cta, L.nrp - 8 * rb0);
-        for (int r = threadIdx.x; r < npairs; r += cthreads) y[8 * rb0 + r] = yout[r];
+    if (gated == 2) {
+        const int4 sh = ctab[0];                        // (first row block, row blocks, first row)
+        const int rows = min(16 * sh.y, J.n[0] - 16 * sh.x);
+        for (int r = threadIdx.x; r < rows; r += cthreads) J.y[0][16 * sh.x + r] = yout[r];
         return;
     }
-    const int rows = min(16 * n_cta, L.n - 16 * rb0);
-    for (int r = threadIdx.x; r < rows; r += cthreads) y[16 * rb0 + r] = yout[r];
+    for (int j = 0; j < njobs; ++j) {
+        const int4 sh = ctab[j];
+        if (gated == 1) {
+            const int npairs = min(8 * sh.y, J.nrp[j] - 8 * sh.x);
+            for (int r = threadIdx.x; r < npairs; r += cthreads) J.y[j][8 * sh.x + r] = yout[sh.z / 2 + r];
+        } else {
+            const int rows = min(16 * sh.y, J.n[j] - 16 * sh.x);
+            for (int r = threadIdx.x; r < rows; r += cthreads) J.y[j][16 * sh.x + r] = yout[sh.z + r];
+        }
+    }
 }
 
-template <int D, int RU>
-ptqtp_status launch_d4(const Layout3& L, const void* packed, const uint16_t* x, uint16_t* y, int grid, int warps,
-                       int rows_cap, size_t smem, int speculate, int gated, cudaStream_t st) {
-    ptqtp_status s = configure_once<gemv4_kernel<D, RU>>();
+template <int D, int RU, bool kMulti>
+ptqtp_status launch_d4(const Jobs4& J, const uint16_t* x, int grid, int warps, int rows_cap, size_t smem, int speculate,
+                       int gated, cudaStream_t st) {
+    ptqtp_status s = configure_once<gemv4_kernel<D, RU, kMulti>>();
     if (s != PTQTP_OK) return s;
     int* status_word = nullptr;                           // shared with the other GEMV kernels (ptqtp_kernel_status)
     if (gemv_status_word(&status_word) != PTQTP_OK) return PTQTP_ERR_CUDA;
@@ -429,9 +503,8 @@ ptqtp_status launch_d4(const Layout3& L, const void* packed, const uint16_t* x, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap_enabled() && !consume_pack(st) ? 1 : 0;   // plain right after a pack on this stream
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv4_kernel<D, RU>, L, static_cast<const unsigned char*>(packed),
-                                       reinterpret_cast<const __half*>(x), reinterpret_cast<__half*>(y), rows_cap,
-                                       L.nrb / grid, L.nrb % grid, speculate, overlap_enabled() ? 1 : 0, gated, wait_poll_limit(),
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv4_kernel<D, RU, kMulti>, J, reinterpret_cast<const __half*>(x), rows_cap, speculate,
+                                       overlap_enabled() ? 1 : 0, gated, wait_poll_limit(),
                                        take_injected_wait_failure() ? 1 : 0, status_word);
     if (e != cudaSuccess) { set_last_cuda_error(e); (void)cudaGetLastError(); return PTQTP_ERR_CUDA; }
     return PTQTP_OK;
@@ -439,13 +512,15 @@ ptqtp_status launch_d4(const Layout3& L, const void* packed, const uint16_t* x, 
 
 }  // namespace
 
-// gated: y[i] = silu(row 2i) * row 2i+1 instead of the rows themselves (N even).
+// jobs: the matrices of the launch (codes, y, n, nrp, nrb, count, k, sbs filled in by the caller; the partition
+// fields are set here).  gated: 0 = the rows themselves; 1 = y[i] = silu(row 2i) * row 2i+1 within every job (N
+// even); 2 = y0[i] = silu(row i of job 0) * row i of job 1 (two jobs of equal shape).
 // warps: per CTA, 0 = the default below, -1 = as many as fit (for a call that is known to run alone).
 // ctas_per_sm: CTAs of this launch per SM (0 = one).  units: tiles per bulk copy (1 or 2; 0 = library choice).
 // depth: copies in flight per warp (2, 3, 4, 6; 0 = library choice).
-ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
-                          int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated) {
-    const int S = L.sbs;
+ptqtp_status launch_gemv4_jobs(Jobs4& J, const uint16_t* x, int warps, int ctas_per_sm, int depth, int units,
+                               cudaStream_t st, int gated) {
+    const int S = J.sbs;
     if (ctas_per_sm < 0 || ctas_per_sm > 4) return PTQTP_ERR_CONFIG;
     if (warps < -1 || warps > kMaxWarps4) return PTQTP_ERR_CONFIG;
     if (units != 0 && units != 1 && units != 2) return PTQTP_ERR_CONFIG;
@@ -453,8 +528,20 @@ ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* 
     const int per_sm = ctas_per_sm ? ctas_per_sm : 1;
     const int max_warps = kMaxWarps4 / per_sm;
     const size_t budget = (size_t)(228 / per_sm - 1) * 1024;          // 228 KB per SM, 1 KB of it reserved per CTA
-    const int grid = min(per_sm * sm_count(), L.nrb);
-    const int rb_cap = (L.nrb + grid - 1) / grid;
+    int total_rb = 0;
+    for (int j = 0; j < J.count; ++j) total_rb += J.nrb[j];
+    const int grid = min(per_sm * sm_count(), total_rb);
+    // every job is spread over the whole grid; the CTAs that take one row block more start, job after job, where
+    // the previous job's stopped, so that the sums differ by one block at most (a gated pair of two jobs keeps
+    // equal partitions: both rows of an output must be in the same CTA)
+    int rb_cap = 0, off = 0;
+    for (int j = 0; j < J.count; ++j) {
+        J.rb_base[j] = J.nrb[j] / grid;
+        J.rb_rem[j] = J.nrb[j] % grid;
+        J.rb_off[j] = gated == 2 ? 0 : off;
+        off = (off + J.rb_rem[j]) % grid;
+        rb_cap += J.rb_base[j] + (J.rb_rem[j] ? 1 : 0);
+    }
     const int rows_cap = 16 * rb_cap;
     const bool alone = warps == -1 || (warps == 0 && !overlap_enabled());   // plain launches never share an SM
     if (warps <= 0) {
@@ -473,14 +560,17 @@ ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* 
     if (auto_depth) depth = alone ? 4 : 2;
     if (auto_units) units = 1;
     if (auto_depth)
-        while (depth > 2 && smem_layout4(L.k, S, rows_cap, warps, depth, units).total > budget) --depth;
+        while (depth > 2 && smem_layout4(J.k, S, rows_cap, warps, depth, units).total > budget) --depth;
     if (depth == 5) depth = 4;
-    const size_t smem = smem_layout4(L.k, S, rows_cap, warps, depth, units).total;
+    const size_t smem = smem_layout4(J.k, S, rows_cap, warps, depth, units).total;
     if (smem > budget) return !auto_depth || !auto_units || ctas_per_sm > 1 || warps > 1 ? PTQTP_ERR_CONFIG : PTQTP_ERR_SHAPE;
-#define PTQTP_LAUNCH_D4(DD)                                                                                      \
-    case DD:                                                                                                     \
-        return units == 1 ? launch_d4<DD, 1>(L, packed, x, y, grid, warps, rows_cap, smem, spec, gated ? 1 : 0, st) \
-                          : launch_d4<DD, 2>(L, packed, x, y, grid, warps, rows_cap, smem, spec, gated ? 1 : 0, st);
+#define PTQTP_LAUNCH_D4(DD)                                                                        \
+    case DD:                                                                                       \
+        if (J.count > 1)                                                                                  \
+            return units == 1 ? launch_d4<DD, 1, true>(J, x, grid, warps, rows_cap, smem, spec, gated, st)   \
+                              : launch_d4<DD, 2, true>(J, x, grid, warps, rows_cap, smem, spec, gated, st);  \
+        return units == 1 ? launch_d4<DD, 1, false>(J, x, grid, warps, rows_cap, smem, spec, gated, st)      \
+                          : launch_d4<DD, 2, false>(J, x, grid, warps, rows_cap, smem, spec, gated, st);
     switch (depth) {
         PTQTP_LAUNCH_D4(2)
         PTQTP_LAUNCH_D4(3)
@@ -489,6 +579,24 @@ ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* 
     }
 #undef PTQTP_LAUNCH_D4
     return PTQTP_ERR_CONFIG;
+}
+
+void add_job4(Jobs4& J, const Layout3& L, const void* packed, uint16_t* y) {
+    const int j = J.count++;
+    J.codes[j] = static_cast<const unsigned char*>(packed) + L.codes_off;
+    J.y[j] = reinterpret_cast<__half*>(y);
+    J.n[j] = L.n;
+    J.nrp[j] = L.nrp;
+    J.nrb[j] = L.nrb;
+    J.k = L.k;
+    J.sbs = L.sbs;
+}
+
+ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
+                          int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated) {
+    Jobs4 J = {};
+    add_job4(J, L, packed, y);
+    return launch_gemv4_jobs(J, x, warps, ctas_per_sm, depth, units, st, gated ? 1 : 0);
 }
 
 }  // namespace ptqtp

@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libptqtp (not part of the ABI).
 #pragma once
 #include <cuda_runtime.h>
+#include <cuda_fp16.h>
 #include <mutex>
 #include <stdint.h>
 #include <stddef.h>
@@ -140,6 +141,18 @@ ptqtp_status launch_pack3(const Layout3& L, const int8_t* T1, const int8_t* T2, 
                           const uint16_t* a2, void* packed, int32_t* dev_status, cudaStream_t st);
 ptqtp_status launch_unpack3(const Layout3& L, const void* packed, int8_t* T1, int8_t* T2, uint16_t* a1,
                             uint16_t* a2, int32_t* dev_status, cudaStream_t st);
+// The matrices ("jobs") of one launch of the format-3 batch-1 kernel: they share x (and therefore K).
+constexpr int kMaxJobs4 = 4;
+struct Jobs4 {
+    const unsigned char* codes[kMaxJobs4];    // first tile of each packed blob
+    ::__half* y[kMaxJobs4];
+    int n[kMaxJobs4], nrp[kMaxJobs4], nrb[kMaxJobs4];
+    int rb_base[kMaxJobs4], rb_rem[kMaxJobs4], rb_off[kMaxJobs4];   // balanced partition of each job over the grid
+    int count, k, sbs;
+};
+void add_job4(Jobs4& J, const Layout3& L, const void* packed, uint16_t* y);
+ptqtp_status launch_gemv4_jobs(Jobs4& J, const uint16_t* x, int warps, int ctas_per_sm, int depth, int units,
+                               cudaStream_t st, int gated);
 // warps: per CTA (0 = library choice, -1 = as many as fit); depth: tiles in flight per warp (0 = library choice)
 ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
                           int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated = false);

@@ -22,13 +22,13 @@ def decode_overlap_level():
 
 
 def _smem_bytes(N, K, warps, depth, units, per_sm):
-    """Shared memory of a launch, from the kernel's layout: x as read (2 K bytes), a staging area of 1088 bytes per
-    warp, the partial sums, the fp16 rows, one mbarrier per ring slot and one for x, the ring (tiles of 4352 bytes)
+    """Shared memory of a launch, from the kernel's layout: x as read (2 K bytes), a staging area of 1120 bytes per
+    warp, the partial sums, the fp16 rows, the table of the CTA's shares (64 bytes), one mbarrier per ring slot and one for x, the ring (tiles of 4352 bytes)
     from a 128-byte boundary."""
     S, nrb = -(-K // 512), -(-((N + 1) // 2) // 8)
     rows_cap = 16 * -(-nrb // min(per_sm * 148, nrb))
-    off = 2 * K + warps * 1088 + rows_cap * S * 4 + rows_cap * 2
-    off = -(-off // 8) * 8 + (warps * depth + 1) * 8
+    off = 2 * K + warps * 1120 + rows_cap * S * 4 + rows_cap * 2
+    off = -(-off // 16) * 16 + 64 + (warps * depth + 1) * 8
     return -(-off // 128) * 128 + warps * depth * units * 4352
 
 
@@ -260,3 +260,59 @@ def test_llama3_8b_shapes_whole_sm_launch(name):
     y = binding.ptqtp_gemv_cfg(pack_case(c, V3), N, K, dev(c["x"]), k_split=-1, fmt=V3)
     torch.cuda.synchronize()
     assert_parity(y.cpu().numpy(), oracle_y(c), c["x"], name)
+
+
+@pytest.mark.parametrize("level", [0, 2])
+@pytest.mark.parametrize("Ns,K", [((4096, 1024, 1024), 4096), ((5, 33, 130, 7), 1152), ((1000,), 2048), ((14336, 14336), 4096),
+                                  ((64, 2400), 14336), ((16, 16, 16, 16), 128)])
+def test_several_matrices_in_one_launch_give_the_bits_of_separate_calls(Ns, K, level):
+    binding.ptqtp_set_overlap(level)
+    cs = [make_case(N, K, seed=500 + 7 * j + N) for j, N in enumerate(Ns)]
+    x = cs[0]["x"]
+    packed = [pack_case(c, V3) for c in cs]
+    ys = binding.ptqtp_gemv_multi(packed, list(Ns), K, dev(x))
+    torch.cuda.synchronize()
+    for j, (c, p, y) in enumerate(zip(cs, packed, ys)):
+        alone = binding.ptqtp_gemv(p, c["N"], K, dev(x), fmt=V3)
+        torch.cuda.synchronize()
+        assert np.array_equal(y.cpu().numpy().view(np.uint16), alone.cpu().numpy().view(np.uint16)), j
+        assert_parity(y.cpu().numpy(), oracle_y(dict(c, x=x)), x, "matrix %d of %s" % (j, Ns))
+
+
+@pytest.mark.parametrize("N,K", [(16, 128), (300, 1152), (14336, 4096), (2401, 2048)])
+def test_gated_pair_of_two_matrices_in_one_launch(N, K):
+    cg, cu = make_case(N, K, seed=600 + N), make_case(N, K, seed=601 + N)
+    cg["alpha1"] = (cg["alpha1"].astype(np.float32) * 4).astype(np.float16)          # gate values of order 1
+    x = cg["x"]
+    (y,) = binding.ptqtp_gemv_multi([pack_case(cg, V3), pack_case(cu, V3)], [N, N], K, dev(x),
+                                    epilogue=binding.EPILOGUE_GATED_PAIR)
+    torch.cuda.synchronize()
+    y = y.cpu().numpy().astype(np.float64)
+    g, u = oracle_y(dict(cg, x=x)), oracle_y(dict(cu, x=x))
+    ref = g / (1.0 + np.exp(-g)) * u
+    B = 2e-3 * float(np.abs(x.astype(np.float64)).max()) * np.sqrt(K)
+    bound = B * (1.1 * np.abs(u) + np.abs(g / (1.0 + np.exp(-g)))) + 2.0 ** -10 * np.abs(ref) + 1e-7
+    assert y.shape == (N,) and np.all(np.isfinite(y))
+    assert np.all(np.abs(y - ref) <= bound)
+    assert np.linalg.norm(y - ref) <= 1e-3 * np.linalg.norm(ref) + 1e-6
+    # the same bits as the interleaved single-matrix form of the epilogue
+    inter = dict(N=2 * N, K=K, x=x, **{k: np.stack([cg[k], cu[k]], axis=1).reshape(2 * N, -1) for k in ("T1", "T2", "alpha1", "alpha2")})
+    yi = binding.ptqtp_gemv_swiglu(pack_case(inter, V3), 2 * N, K, dev(x), fmt=V3)
+    torch.cuda.synchronize()
+    assert np.array_equal(yi.cpu().numpy().astype(np.float64), y)
+
+
+def test_several_matrices_argument_checks():
+    K = 1024
+    cs = [make_case(64, K, seed=1), make_case(32, K, seed=2)]
+    p3 = [pack_case(c, V3) for c in cs]
+    x = dev(cs[0]["x"])
+    with pytest.raises(binding.PtqtpError) as e:             # gated pair needs equal N
+        binding.ptqtp_gemv_multi(p3, [64, 32], K, x, epilogue=binding.EPILOGUE_GATED_PAIR)
+    assert e.value.status == binding.ERR_SHAPE
+    with pytest.raises(binding.PtqtpError) as e:             # more than four matrices
+        binding.ptqtp_gemv_multi([p3[0]] * 5, [64] * 5, K, x)
+    assert e.value.status == binding.ERR_SHAPE
+    with pytest.raises(binding.PtqtpError) as e:
+        binding.ptqtp_gemv_multi(p3, [64, 32], K, x, epilogue=7)
+    assert e.value.status == binding.ERR_CONFIG
