@@ -234,6 +234,43 @@ PTQTP_API ptqtp_status ptqtp_gemm_skinny_static(const ptqtp_shape *shape /* host
                                       size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                       void *stream);
 
+/* Progressive trit-plane decomposition on the GPU: W [n, k] (device, fp32, row-major) -> planes T1, T2 (device int8
+ * [n*k], entries in {-1,0,1}) and scales alpha1, alpha2 (device fp16 bits [n*k/group]) with
+ * W ~ alpha1 (.) T1 + alpha2 (.) T2 per group-row -- the step before ptqtp_pack.  Algorithm 1 (group-rows, sweeps,
+ * stop when the largest change of a scale pair over all group-rows is below eps or after t_max sweeps) with the
+ * inner formulas of Algorithm 2 and Appendix C: initial planes sign(w) (0 -> +1), alpha = (1, 1), lambda = 1e-8;
+ * ridge solve of Eq. 3-5 by the explicit 2 x 2 inverse; kappa = ||A||_F ||A^-1||_F (Eq. 6), and when kappa >= 1e6
+ * lambda <- min(lambda sqrt(kappa / 1e6), 1), used by the same sweep's solve; per element the pair in {-1,0,1}^2
+ * of smallest squared error, equal errors resolved towards fewer non-zeros, then towards plane 1.  The returned
+ * iterate is (alpha_t, T_t) of the last sweep, without a refit.  canonicalize != 0: afterwards, per group-row and
+ * without changing alpha1 T1 + alpha2 T2, both scales are made non-negative (flipping plane and scale) and ordered
+ * alpha1 >= alpha2 (exchanging the planes).  The scales are rounded to fp16 once, at the end.
+ * Arithmetic: IEEE double precision, every operation rounded on its own, sums in column order: a run is
+ * reproducible bit for bit.  group: 1..PTQTP_DECOMPOSE_MAX_GROUP, k % group == 0 (ptqtp_pack needs group = 128);
+ * t_max: 1..PTQTP_DECOMPOSE_MAX_SWEEPS (the paper uses 50, eps = 1e-4).
+ * workspace: device, 16-byte aligned, ptqtp_decompose_workspace_size bytes, contents irrelevant on entry.  On
+ * return (after syncing) it holds, at the offsets given by ptqtp_decompose_layout: int32 sweeps run; per sweep
+ * t = 1..sweeps the largest change of a scale pair (f64 at delta_offset + 8 t) and the total squared error after the
+ * sweep (f64 at error_offset + 8 (t - 1)); per group-row the unrounded scales and lambda (f64).
+ * 2 t_max + 2 small kernels are enqueued on `stream`; no synchronisation. */
+#define PTQTP_DECOMPOSE_MAX_GROUP 256
+#define PTQTP_DECOMPOSE_MAX_SWEEPS 1000
+typedef struct {
+    size_t sweeps_offset;   /* int32 */
+    size_t delta_offset;    /* f64 [t_max + 1], entry t for sweep t */
+    size_t error_offset;    /* f64 [t_max] */
+    size_t alpha1_offset;   /* f64 [n * k / group] */
+    size_t alpha2_offset;   /* f64 [n * k / group] */
+    size_t lambda_offset;   /* f64 [n * k / group] */
+    size_t total_bytes;
+} ptqtp_decompose_offsets;
+PTQTP_API size_t ptqtp_decompose_workspace_size(int32_t n, int32_t k, int32_t group, int32_t t_max);
+PTQTP_API ptqtp_status ptqtp_decompose_layout(int32_t n, int32_t k, int32_t group, int32_t t_max,
+                                    ptqtp_decompose_offsets *out /* host */);
+PTQTP_API ptqtp_status ptqtp_decompose(const float *W, int32_t n, int32_t k, int32_t group, int32_t t_max, double eps,
+                             int32_t canonicalize, int8_t *T1, int8_t *T2, uint16_t *alpha1, uint16_t *alpha2,
+                             void *workspace, size_t workspace_bytes, void *stream);
+
 /* End-to-end convenience for callers holding activations on the host: copies x_host [K] (host,
  * ideally pinned) to x_dev, runs ptqtp_gemv and delivers y in y_host [N]; everything is enqueued on
  * `stream`, no synchronisation: y_host is valid once the stream has reached this point.  x_dev [K] and

@@ -26,7 +26,8 @@ EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptq
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
            "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws",
            "ptqtp_gemm_skinny_static", "ptqtp_kernel_status", "ptqtp_gemv_swiglu", "ptqtp_kernel_status_clear",
-           "ptqtp_set_wait_limit", "ptqtp_test_fail_next_wait", "ptqtp_gemv_multi")
+           "ptqtp_set_wait_limit", "ptqtp_test_fail_next_wait", "ptqtp_gemv_multi", "ptqtp_decompose",
+           "ptqtp_decompose_workspace_size", "ptqtp_decompose_layout")
 
 
 class PtqtpError(RuntimeError):
@@ -34,6 +35,11 @@ class PtqtpError(RuntimeError):
         self.status = status
         super().__init__("%s failed: %s (status %d, cuda error %d)"
                          % (what, status_string(status), status, lib().ptqtp_last_cuda_error()))
+
+
+class DecomposeOffsets(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_size_t) for n in ("sweeps_offset", "delta_offset", "error_offset", "alpha1_offset",
+                                               "alpha2_offset", "lambda_offset", "total_bytes")]
 
 
 class Shape(ctypes.Structure):
@@ -64,6 +70,12 @@ def lib():
         L.ptqtp_gemv.argtypes = [sp, vp, sz, vp, vp, vp]
         L.ptqtp_gemv_swiglu.restype = ctypes.c_int
         L.ptqtp_gemv_swiglu.argtypes = [sp, vp, sz, vp, vp, vp]
+        L.ptqtp_decompose_workspace_size.restype = sz
+        L.ptqtp_decompose_workspace_size.argtypes = [i32, i32, i32, i32]
+        L.ptqtp_decompose_layout.restype = ctypes.c_int
+        L.ptqtp_decompose_layout.argtypes = [i32, i32, i32, i32, ctypes.POINTER(DecomposeOffsets)]
+        L.ptqtp_decompose.restype = ctypes.c_int
+        L.ptqtp_decompose.argtypes = [vp, i32, i32, i32, i32, ctypes.c_double, i32, vp, vp, vp, vp, vp, sz, vp]
         L.ptqtp_gemv_multi.restype = ctypes.c_int
         L.ptqtp_gemv_multi.argtypes = [i32, sp, ctypes.POINTER(vp), ctypes.POINTER(sz), vp, ctypes.POINTER(vp), i32, vp]
         L.ptqtp_gemm_skinny.restype = ctypes.c_int
@@ -199,6 +211,40 @@ def ptqtp_gemv_swiglu(packed, N, K, x, y=None, stream=None, fmt=FORMAT_V2):
                                  _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"), _stream_ptr(stream))
     _check(st, "ptqtp_gemv_swiglu")
     return y
+
+
+def ptqtp_decompose(W, group=GROUP, t_max=50, eps=1e-4, canonicalize=True, stream=None, details=False):
+    """Trit-plane decomposition of a CUDA fp32 matrix W [N, K] on the GPU.  Returns (T1, T2, alpha1, alpha2) as CUDA
+    tensors (int8 planes, fp16 scales [N, K/group]); with details=True also a dict with the number of sweeps, the
+    per-sweep largest scale change and total squared error, and the unrounded fp64 scales (synchronises)."""
+    N, K = W.shape
+    need = int(lib().ptqtp_decompose_workspace_size(N, K, int(group), int(t_max)))
+    if need == 0:
+        raise PtqtpError(ERR_SHAPE, "ptqtp_decompose_workspace_size")
+    dev = W.device
+    ws = torch.empty(need, dtype=torch.uint8, device=dev)
+    T1 = torch.empty((N, K), dtype=torch.int8, device=dev)
+    T2 = torch.empty((N, K), dtype=torch.int8, device=dev)
+    a1 = torch.empty((N, K // group), dtype=torch.float16, device=dev)
+    a2 = torch.empty((N, K // group), dtype=torch.float16, device=dev)
+    st = lib().ptqtp_decompose(_dev(W, torch.float32, "W"), N, K, int(group), int(t_max), float(eps), int(bool(canonicalize)),
+                               _dev(T1, torch.int8, "T1"), _dev(T2, torch.int8, "T2"), _dev(a1, torch.float16, "alpha1"),
+                               _dev(a2, torch.float16, "alpha2"), _dev(ws, torch.uint8, "workspace"), ws.numel(),
+                               _stream_ptr(stream))
+    _check(st, "ptqtp_decompose")
+    if not details:
+        return T1, T2, a1, a2
+    off = DecomposeOffsets()
+    _check(lib().ptqtp_decompose_layout(N, K, int(group), int(t_max), ctypes.byref(off)), "ptqtp_decompose_layout")
+    (stream or torch.cuda.current_stream()).synchronize()
+    host = ws.cpu().numpy()
+    R = N * (K // group)
+    sweeps = int(host[off.sweeps_offset:off.sweeps_offset + 4].view("<i4")[0])
+    f64 = lambda o, n: host[o:o + 8 * n].view("<f8").copy()
+    info = dict(sweeps=sweeps, delta_history=f64(off.delta_offset + 8, sweeps), err_history=f64(off.error_offset, sweeps),
+                alpha1=f64(off.alpha1_offset, R).reshape(N, K // group), alpha2=f64(off.alpha2_offset, R).reshape(N, K // group),
+                lam=f64(off.lambda_offset, R).reshape(N, K // group))
+    return T1, T2, a1, a2, info
 
 
 EPILOGUE_NONE, EPILOGUE_GATED_PAIR = 0, 1

@@ -191,6 +191,38 @@ ptqtp_status ptqtp_gemv_swiglu(const ptqtp_shape* shape, const void* packed, siz
     return launch_gemv2(L.l2, packed, x, y, 0, 0, 0, 0, static_cast<cudaStream_t>(stream), true);
 }
 
+static bool decompose_args_ok(int32_t n, int32_t k, int32_t group, int32_t t_max) {
+    return n > 0 && k > 0 && group >= 1 && group <= PTQTP_DECOMPOSE_MAX_GROUP && k % group == 0 && t_max >= 1 &&
+           t_max <= PTQTP_DECOMPOSE_MAX_SWEEPS;
+}
+
+size_t ptqtp_decompose_workspace_size(int32_t n, int32_t k, int32_t group, int32_t t_max) {
+    if (!decompose_args_ok(n, k, group, t_max)) return 0;
+    return decompose_workspace_bytes((long long)n * (k / group), t_max);
+}
+
+ptqtp_status ptqtp_decompose_layout(int32_t n, int32_t k, int32_t group, int32_t t_max, ptqtp_decompose_offsets* out) {
+    if (!out) return PTQTP_ERR_NULL;
+    if (!decompose_args_ok(n, k, group, t_max)) return PTQTP_ERR_SHAPE;
+    out->sweeps_offset = 0;
+    decompose_offsets((long long)n * (k / group), t_max, &out->delta_offset, &out->error_offset, &out->alpha1_offset,
+                      &out->alpha2_offset, &out->lambda_offset);
+    out->total_bytes = decompose_workspace_bytes((long long)n * (k / group), t_max);
+    return PTQTP_OK;
+}
+
+ptqtp_status ptqtp_decompose(const float* W, int32_t n, int32_t k, int32_t group, int32_t t_max, double eps,
+                             int32_t canonicalize, int8_t* T1, int8_t* T2, uint16_t* alpha1, uint16_t* alpha2,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    if (!W || !T1 || !T2 || !alpha1 || !alpha2 || !workspace) return PTQTP_ERR_NULL;
+    if (!decompose_args_ok(n, k, group, t_max) || !(eps >= 0.0)) return PTQTP_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(T1) || !aligned16(T2) || !aligned16(alpha1) || !aligned16(alpha2) || !aligned16(workspace))
+        return PTQTP_ERR_ALIGN;
+    if (workspace_bytes < decompose_workspace_bytes((long long)n * (k / group), t_max)) return PTQTP_ERR_SIZE;
+    return launch_decompose(W, n, k, group, t_max, eps, canonicalize ? 1 : 0, T1, T2, alpha1, alpha2, workspace,
+                            static_cast<cudaStream_t>(stream));
+}
+
 ptqtp_status ptqtp_gemv_multi(int32_t count, const ptqtp_shape* shapes, const void* const* packed,
                               const size_t* packed_bytes, const uint16_t* x, uint16_t* const* y, int32_t epilogue,
                               void* stream) {

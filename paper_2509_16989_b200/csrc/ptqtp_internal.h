@@ -156,6 +156,11 @@ ptqtp_status launch_gemv4_jobs(Jobs4& J, const uint16_t* x, int warps, int ctas_
 // warps: per CTA (0 = library choice, -1 = as many as fit); depth: tiles in flight per warp (0 = library choice)
 ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
                           int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated = false);
+size_t decompose_workspace_bytes(long long rows, int t_max);
+void decompose_offsets(long long rows, int t_max, size_t* delta_off, size_t* err_off, size_t* a1_off, size_t* a2_off,
+                       size_t* lam_off);
+ptqtp_status launch_decompose(const float* W, int n, int k, int G, int t_max, double eps, int canonicalize, int8_t* T1,
+                              int8_t* T2, uint16_t* alpha1, uint16_t* alpha2, void* workspace, cudaStream_t st);
 size_t skinny3_workspace_bytes(int k, int m);
 ptqtp_status launch_skinny3(const Layout2& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, void* workspace,
                             cudaStream_t st);

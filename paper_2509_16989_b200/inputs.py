@@ -56,3 +56,14 @@ def make_activations(K, seed=0, M=1):
     rng = np.random.default_rng(seed)
     shape = (K,) if M == 1 else (M, K)
     return rng.standard_normal(shape, dtype=np.float32).astype(np.float16)
+
+
+def make_weights_device(N, K, seed=0, sigma=0.02, outlier_frac=1e-3, outlier_gain=20.0, device="cuda"):
+    """The same distribution as make_weights, drawn on the device with torch's generator (for workloads that are
+    too large to draw on the host: each entry is an outlier with probability outlier_frac, independently)."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    W = torch.randn((N, K), generator=g, device=device, dtype=torch.float32) * sigma
+    mask = torch.rand((N, K), generator=g, device=device) < outlier_frac
+    return torch.where(mask, W * outlier_gain, W).contiguous()

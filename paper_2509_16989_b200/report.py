@@ -13,10 +13,11 @@ a decoder would whose packed blobs never change while GEMV calls are in flight.
      28672 x 4096 matrix (rows are independent, so a caller may stack matrices that share their input and
      slice y): five or four calls per layer instead of seven
   6  the seven linears of a LLaMA-3-70B-shaped layer as one chain of calls
-
-(The 32-layer stack built from decomposed weights needs planes from the decomposition of Algorithm 1, which this
-package does not contain; tests/test_gpu_stack.py builds it with the CPU oracle and checks parity on it.  Its
-timing per layer is that of the benchmark's step: the kernels are branch-free in the plane values.)
+  4  the 32-layer stack of LLaMA-3-8B-shaped linears from decomposed weights: W ~ N(0, 0.02^2) with 0.1 % of the
+     entries times 20, drawn on the device, 224 distinct matrices decomposed by ptqtp_decompose and packed; one decode
+     step = 224 calls in one CUDA graph; reports the time per token, the decomposition time and the reconstruction
+     error ||W - (alpha1 T1 + alpha2 T2)||_F / ||W||_F per matrix type (tests/test_gpu_stack.py checks parity of
+     such a stack against the CPU oracle)
 
 Every timing is a CUDA-event steady state inside a CUDA graph that walks over distinct packed buffers
 totalling more than twice the L2 size, so the planes come from HBM.  One JSON line per result.
@@ -34,7 +35,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 from paper_2509_16989_b200 import binding  # noqa: E402
-from paper_2509_16989_b200.inputs import LLAMA3_8B, LLAMA3_70B, QWEN3_0P6B_UP, make_case  # noqa: E402
+from paper_2509_16989_b200.inputs import LLAMA3_8B, LLAMA3_70B, QWEN3_0P6B_UP, make_case, make_weights_device  # noqa: E402
 
 FMT = binding.FORMAT_V3          # packed format of the batch-1 calls (--format)
 
@@ -206,10 +207,49 @@ def config6(T):
          gbs=round(nb / us / 1e3, 1), bytes=nb, layer_copies=2)
 
 
+def config4(T, layers=32):
+    names = ("q", "k", "v", "o", "gate", "up", "down")
+    stack, err2, w2, sweeps = [], {m: 0.0 for m in names}, {m: 0.0 for m in names}, []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dec_ms = 0.0
+    for l in range(layers):
+        layer = {}
+        for mi, m in enumerate(names):
+            N, K = LLAMA3_8B[m]
+            W = make_weights_device(N, K, seed=1000 + 7 * l + mi)
+            torch.cuda.synchronize()
+            e0.record()
+            T1, T2, a1, a2, info = binding.ptqtp_decompose(W, details=True)
+            e1.record()
+            torch.cuda.synchronize()
+            dec_ms += e0.elapsed_time(e1)
+            sweeps.append(info["sweeps"])
+            layer[m], st = binding.ptqtp_pack(T1, T2, a1, a2, fmt=FMT)
+            # reconstruction error with the fp16 scales that were packed (plain torch arithmetic on the device)
+            What = (a1.float().repeat_interleave(128, dim=1) * T1.float() + a2.float().repeat_interleave(128, dim=1) * T2.float())
+            err2[m] += float(((W - What).double() ** 2).sum())
+            w2[m] += float((W.double() ** 2).sum())
+            del W, What, T1, T2, a1, a2
+        stack.append(layer)
+    xs = {m: torch.randn(LLAMA3_8B[m][1], device="cuda").half() for m in names}
+    ys = {m: torch.empty(LLAMA3_8B[m][0], dtype=torch.float16, device="cuda") for m in names}
+    calls = [lambda p=layer[m], m=m: binding.ptqtp_gemv(p, *LLAMA3_8B[m], xs[m], y=ys[m], stream=T.stream, fmt=FMT)
+             for layer in stack for m in names]
+    us = T.steady_us(calls, reps=20) * len(calls)
+    nb = layers * sum(algorithmic_bytes(*LLAMA3_8B[m]) for m in names)
+    emit(workload="cfg4 %d-layer llama3-8b linear stack, weights decomposed on the GPU, batch 1" % layers,
+         call="%d x ptqtp_gemv (format %d)" % (len(calls), FMT), us_per_token=round(us, 1), us_per_layer=round(us / layers, 3),
+         gbs=round(nb / us / 1e3, 1), bytes=nb, distinct_decomposed_layers=layers,
+         reconstruction_error={m: round((err2[m] / w2[m]) ** 0.5, 4) for m in names},
+         reconstruction_error_all=round((sum(err2.values()) / sum(w2.values())) ** 0.5, 4),
+         decompose_ms_total=round(dec_ms, 1), decompose_ms_per_layer=round(dec_ms / layers, 2),
+         sweeps_min=int(min(sweeps)), sweeps_max=int(max(sweeps)))
+
+
 def main():
     global FMT
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="0,2,3,5,6")
+    ap.add_argument("--only", default="0,2,3,4,5,6")
     ap.add_argument("--format", type=int, default=3, choices=(2, 3))
     args = ap.parse_args()
     if not torch.cuda.is_available():
@@ -229,6 +269,8 @@ def main():
         config5(T)
     if 6 in which:
         config6(T)
+    if 4 in which:
+        config4(T)
 
 
 

@@ -123,6 +123,24 @@ def test_host_side_validation_codes(L):
         assert L.ptqtp_gemm_skinny_workspace_size(ctypes.byref(sh), 2) == 0
 
 
+def test_decompose_host_side_checks(L):
+    ok_ptr, odd_ptr = ctypes.c_void_p(0x10000), ctypes.c_void_p(0x10008)
+    need = L.ptqtp_decompose_workspace_size(8, 256, 128, 50)
+    off = binding.DecomposeOffsets()
+    assert L.ptqtp_decompose_layout(8, 256, 128, 50, ctypes.byref(off)) == binding.OK
+    assert off.total_bytes == need and off.sweeps_offset == 0 and off.delta_offset == 64
+    assert off.error_offset == 64 + 51 * 8 and off.alpha2_offset - off.alpha1_offset == 16 * 8
+    assert off.lambda_offset + 16 * 8 == need
+    assert L.ptqtp_decompose_layout(8, 250, 128, 50, ctypes.byref(off)) == binding.ERR_SHAPE
+    args = lambda **kw: [kw.get("W", ok_ptr), 8, kw.get("k", 256), 128, 50, ctypes.c_double(kw.get("eps", 1e-4)), 1, ok_ptr, ok_ptr,
+                         kw.get("a1", ok_ptr), ok_ptr, ok_ptr, kw.get("size", need), None]
+    assert L.ptqtp_decompose(*args(W=None)) == binding.ERR_NULL
+    assert L.ptqtp_decompose(*args(k=200)) == binding.ERR_SHAPE
+    assert L.ptqtp_decompose(*args(eps=-1.0)) == binding.ERR_SHAPE
+    assert L.ptqtp_decompose(*args(a1=odd_ptr)) == binding.ERR_ALIGN
+    assert L.ptqtp_decompose(*args(size=need - 1)) == binding.ERR_SIZE
+
+
 def test_process_wide_settings_defaults_and_setters(L):
     # plain launches are the default: every buffer, the packed blob included, follows stream order
     assert L.ptqtp_set_overlap(1) == 0
