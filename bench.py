@@ -506,8 +506,9 @@ def run_gpu(args):
             # The layer as a decoder issues it: every call's x is written on the stream directly before it is used.
             #   x_q = f(y_down of the layer before); x_k = x_v = x_q; x_o = f(y_q); x_gate = x_up = f(y_o);
             #   x_down = y_gate * y_up   (f = one elementwise kernel, standing in for attention / norms)
-            # 7 GEMV calls + 4 elementwise kernels per layer.  The speculative pass of q, o, gate and down runs on
-            # activations that are rewritten under it and is repeated; k, v and up keep theirs.
+            # 7 GEMV calls + 4 elementwise kernels per layer.  k, v and up start early under their speculative pass; a
+            # call behind an elementwise kernel starts when that kernel has finished (it releases its dependents only
+            # at its end), so q, o, gate and down run alone on the GPU.
             xd = {"a": torch.zeros(4096, dtype=torch.float16, device=device),
                   "o": torch.zeros(4096, dtype=torch.float16, device=device),
                   "m": torch.zeros(4096, dtype=torch.float16, device=device),
@@ -536,17 +537,18 @@ def run_gpu(args):
             detail["step_dependent"] = {
                 "us_per_layer": 1e3 * chain.time_ms([gd] * 10) / (10 * 4 * R),
                 "what": "7 ptqtp_gemv + 4 elementwise kernels per layer; every x is produced on the stream directly "
-                        "before its first use (q, o, gate, down repeat their speculative pass)"}
-            old_level = binding.ptqtp_set_overlap(1)
-            try:
-                with torch.cuda.stream(stream):
-                    dep_layer(0)
-                    stream.synchronize()
-                gd1 = chain.capture(dep_steps)
-                detail["step_dependent"]["us_per_layer_level1"] = 1e3 * chain.time_ms([gd1] * 10) / (10 * 4 * R)
-                del gd1
-            finally:
-                binding.ptqtp_set_overlap(old_level)
+                        "before its first use (q, o, gate, down start only when the elementwise kernel ahead of them has ended)"}
+            for lvl in (1, 0):
+                old_level = binding.ptqtp_set_overlap(lvl)
+                try:
+                    with torch.cuda.stream(stream):
+                        dep_layer(0)
+                        stream.synchronize()
+                    gd1 = chain.capture(dep_steps)
+                    detail["step_dependent"]["us_per_layer_level%d" % lvl] = 1e3 * chain.time_ms([gd1] * 10) / (10 * 4 * R)
+                    del gd1
+                finally:
+                    binding.ptqtp_set_overlap(old_level)
             del gd
             # Four launches per layer (format 3): q, k, v in one launch and gate, up with the gated pair epilogue in
             # one launch (ptqtp_gemv_multi over the separately packed blobs), o and down as before.  First with
