@@ -40,8 +40,9 @@ MATRICES = ("q", "k", "v", "o", "gate", "up", "down")
 UNIQUE_OF = {"q": "qo", "o": "qo", "k": "kv", "v": "kv", "gate": "gate_up", "up": "gate_up", "down": "down"}
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch in the ncu captures of the current batch-1 kernel, one
-# launch per shape (profiles/gemv4_*.md); None for a shape whose kernel has changed since its capture
-DRAM_TRAFFIC_BYTES = {3: {"qo": None, "kv": None, "gate_up": None, "down": None},
+# launch per shape (profiles/gemv4_llama3_8b_shapes.md, profiles/gemv2_gate_up_14336x4096.md); None where no capture
+# of the current kernel exists
+DRAM_TRAFFIC_BYTES = {3: {"qo": 8958720.0, "kv": 2274048.0, "gate_up": 31241216.0, "down": 31261440.0},
                       2: {"qo": None, "kv": None, "gate_up": 31239424.0, "down": None}}
 KERNEL_NAME = {2: "gemv2_kernel", 3: "gemv4_kernel"}
 DTYPE = {2: "int16 block-fixed-point x int2 codes -> int32 (dp4a), f32 scale epilogue",
