@@ -194,8 +194,11 @@ PTQTP_API ptqtp_status ptqtp_gemv_multi(int32_t count, const ptqtp_shape *shapes
  * one pass over the planes at about the cost of a batch-1 call (the activations stay in registers); larger M
  * take one such pass per four rows (ptqtp_gemm_skinny_ws reads the planes once for any M).  When four rows of x
  * leave no room in shared memory (very long K) the passes take three or two rows, or one row on the batch-1
- * kernel.  M = 1 runs the batch-1 kernel.  Formats 1 and 3 are batch-1 layouts: M = 1 runs their batch-1 kernel,
- * M > 1 returns PTQTP_ERR_CONFIG (pack a format-2 blob for small batches). */
+ * kernel.  M = 1 runs the batch-1 kernel.  Format 3: the same tiles and decode as its batch-1 kernel, with the MMA
+ * columns holding two or four batch rows instead of the four scale groups (two or four times the tensor-core work
+ * of one row, the same masks and the same stream of tiles); M = 2 takes one pass at about 1.3 times the cost of a
+ * batch-1 call, larger M take a pass per four rows (two when four rows of x leave no room in shared memory); format
+ * 2 is the faster small-batch layout from M = 3 on.  Format 1 is a batch-1 layout: M > 1 returns PTQTP_ERR_CONFIG. */
 PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, const void *packed,
                                size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                void *stream);
@@ -206,7 +209,7 @@ PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, co
  * converted once to block fixed point; with it the packed planes are read from HBM exactly once for any M and
  * K, where ptqtp_gemm_skinny needs several passes when M or K is large.  Two kernels are enqueued on `stream`.
  * Calls that share a workspace must not overlap on the GPU.  ptqtp_gemm_skinny_workspace_size returns 0 for a
- * bad shape, formats 1 and 3 or M out of range.  (Small-batch use of the layer of Eq. 1-2; the paper measures batch 1.) */
+ * bad shape, formats 1 and 3 (the workspace kernels read format 2) or M out of range.  (Small-batch use of the layer of Eq. 1-2; the paper measures batch 1.) */
 PTQTP_API size_t ptqtp_gemm_skinny_workspace_size(const ptqtp_shape *shape /* host */, int32_t m);
 PTQTP_API ptqtp_status ptqtp_gemm_skinny_ws(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
                                   int32_t m, const uint16_t *X, uint16_t *Y, void *workspace,

@@ -277,7 +277,25 @@ ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, siz
         }
         return launch_gemv2(L.l2, packed, X, Y, 0, 0, 0, 0, st);
     }
-    // formats 1 and 3 are batch-1 layouts: the small-batch kernels read format 2
+    if (L.v3) {
+        // Format 3: up to four rows per pass over the planes on the tensor-core kernel whose MMA columns are the rows
+        // (two rows cost about a batch-1 pass, four about one and a half); more rows take a pass per four, and when
+        // four rows of x leave no room in shared memory the passes take two rows, or one on the batch-1 kernel.
+        int per_pass = m < 4 ? m : 4;
+        int done = 0;
+        while (done < m) {
+            const uint16_t* Xp = X + (size_t)done * shape->k_in;
+            uint16_t* Yp = Y + (size_t)done * shape->n_out;
+            const int rows = m - done < per_pass ? m - done : per_pass;
+            ptqtp_status sp = rows == 1 ? launch_gemv4(L.l3, packed, Xp, Yp, 0, 0, 0, 0, st)
+                                        : launch_gemv5(L.l3, packed, rows, Xp, Yp, 0, 0, st);
+            if (sp == PTQTP_ERR_SHAPE && rows > 1 && done == 0) { per_pass = per_pass > 2 ? 2 : 1; continue; }   // nothing launched yet
+            if (sp != PTQTP_OK) return sp;
+            done += rows;
+        }
+        return PTQTP_OK;
+    }
+    // format 1 is a batch-1 layout
     if (m != 1) return PTQTP_ERR_CONFIG;
     return gemv_any(L, packed, X, Y, 0, 0, 0, 0, -1, st);
 }

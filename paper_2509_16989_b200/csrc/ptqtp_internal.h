@@ -156,6 +156,9 @@ ptqtp_status launch_gemv4_jobs(Jobs4& J, const uint16_t* x, int warps, int ctas_
 // warps: per CTA (0 = library choice, -1 = as many as fit); depth: tiles in flight per warp (0 = library choice)
 ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* x, uint16_t* y, int warps,
                           int ctas_per_sm, int depth, int units, cudaStream_t st, bool gated = false);
+// 2 <= m <= 4 rows on format 3; PTQTP_ERR_SHAPE when (K, m) leaves no room in shared memory
+ptqtp_status launch_gemv5(const Layout3& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, int warps, int depth,
+                          cudaStream_t st);
 size_t decompose_workspace_bytes(long long rows, int t_max);
 void decompose_offsets(long long rows, int t_max, size_t* delta_off, size_t* err_off, size_t* a1_off, size_t* a2_off,
                        size_t* lam_off);

@@ -114,11 +114,12 @@ def test_host_side_validation_codes(L):
     v1 = binding.make_shape(8, 256, fmt=binding.FORMAT_V1)
     assert L.ptqtp_gemv_swiglu(ctypes.byref(v1), ok_ptr, binding.packed_size(8, 256, fmt=binding.FORMAT_V1), ok_ptr, ok_ptr,
                                None) == binding.ERR_CONFIG
-    # formats 1 and 3 are batch-1 layouts: the small-batch calls refuse them for M > 1
+    # format 1 is a batch-1 layout; the workspace calls read format 2 only
     for fmt in (binding.FORMAT_V1, binding.FORMAT_V3):
         sh = binding.make_shape(8, 256, fmt=fmt)
         sz = binding.packed_size(8, 256, fmt=fmt)
-        assert L.ptqtp_gemm_skinny(ctypes.byref(sh), ok_ptr, sz, 2, ok_ptr, ok_ptr, None) == binding.ERR_CONFIG
+        if fmt == binding.FORMAT_V1:
+            assert L.ptqtp_gemm_skinny(ctypes.byref(sh), ok_ptr, sz, 2, ok_ptr, ok_ptr, None) == binding.ERR_CONFIG
         assert L.ptqtp_gemm_skinny_ws(ctypes.byref(sh), ok_ptr, sz, 2, ok_ptr, ok_ptr, ok_ptr, 1 << 20, None) == binding.ERR_CONFIG
         assert L.ptqtp_gemm_skinny_workspace_size(ctypes.byref(sh), 2) == 0
 

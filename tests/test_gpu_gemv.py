@@ -381,7 +381,7 @@ def test_gemm_skinny_matches_oracle_per_row(M, fmt):
     c = make_case(192, 3072, seed=20 + M, M=M)
     packed = pack_case(c, fmt)
     X = dev(np.atleast_2d(c["x"]))
-    if fmt != binding.FORMAT_V2 and M > 1:               # formats 1 and 3 are batch-1 layouts
+    if fmt == binding.FORMAT_V1 and M > 1:               # format 1 is a batch-1 layout
         with pytest.raises(binding.PtqtpError) as e:
             binding.ptqtp_gemm_skinny(packed, 192, 3072, X, fmt=fmt)
         assert e.value.status == binding.ERR_CONFIG

@@ -316,3 +316,33 @@ def test_several_matrices_argument_checks():
     with pytest.raises(binding.PtqtpError) as e:
         binding.ptqtp_gemv_multi(p3, [64, 32], K, x, epilogue=7)
     assert e.value.status == binding.ERR_CONFIG
+
+
+@pytest.mark.parametrize("level", [0, 2])
+@pytest.mark.parametrize("N,K,M", [(1, 128, 2), (5, 256, 3), (7, 1152, 4), (33, 2048, 2), (130, 3200, 4), (257, 5120, 3),
+                                   (64, 14336, 4), (1000, 6144, 7), (37, 36864, 4), (192, 3072, 64), (2400, 4096, 9),
+                                   (14336, 4096, 2), (4096, 14336, 4), (1024, 4096, 3), (4096, 4096, 8)])
+def test_small_batch_on_the_batch1_layout(N, K, M, level):
+    # ptqtp_gemm_skinny on format 3: passes of up to four rows on the kernel whose MMA columns are the batch rows
+    binding.ptqtp_set_overlap(level)
+    c = make_case(N, K, seed=700 + N + M, M=M)
+    packed = pack_case(c, V3)
+    Y = binding.ptqtp_gemm_skinny(packed, N, K, dev(c["x"]), fmt=V3)
+    torch.cuda.synchronize()
+    assert_parity(Y.cpu().numpy(), np.atleast_2d(oracle_y(c)), c["x"], "N=%d K=%d M=%d" % (N, K, M))
+    assert binding.ptqtp_kernel_status() == 0
+
+
+def test_small_batch_on_the_batch1_layout_is_exact_on_integers():
+    N, K, M = 96, 4096, 4
+    c = make_case(N, K, seed=13, M=M)
+    rng = np.random.default_rng(4)
+    c["x"] = rng.integers(-3, 4, (M, K)).astype(np.float16)
+    c["alpha1"] = np.ones_like(c["alpha1"])
+    c["alpha2"] = np.full_like(c["alpha2"], 2.0)
+    exact = (c["x"].astype(np.int64) @ c["T1"].astype(np.int64).T) + 2 * (c["x"].astype(np.int64) @ c["T2"].astype(np.int64).T)
+    assert np.all(np.abs(exact) < 2048)
+    for m in (2, 3, 4):
+        Y = binding.ptqtp_gemm_skinny(pack_case(c, V3), N, K, dev(c["x"][:m].copy()), fmt=V3)
+        torch.cuda.synchronize()
+        assert np.array_equal(Y.cpu().numpy().astype(np.int64), exact[:m]), m
