@@ -203,6 +203,15 @@ PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, co
                                size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                void *stream);
 
+/* ptqtp_gemm_skinny on format 3 with the kernel chosen by the caller (tuning and tests; PTQTP_ERR_CONFIG for the
+ * other formats).  path: 0 = library choice, 5 = passes of up to four rows on the warp-MMA kernel, 6 = the tcgen05
+ * kernel (all M rows in one pass over the planes; fp16 trits from tensor memory against the fp16 activations, fp32
+ * accumulators in tensor memory, fp32 scale epilogue).  k_split (path 6): CTAs of a cluster that share the columns
+ * of a block of 128 rows: 1, 2, 4 or 8; 0 = library choice.  Same result definition as ptqtp_gemm_skinny. */
+PTQTP_API ptqtp_status ptqtp_gemm_skinny_cfg(const ptqtp_shape *shape /* host */, const void *packed, size_t packed_bytes,
+                                   int32_t m, const uint16_t *X, uint16_t *Y, int32_t path, int32_t k_split,
+                                   void *stream);
+
 /* Small-batch variant with a caller-provided workspace (format 2 only; PTQTP_ERR_CONFIG for format 1).
  * Same result definition as ptqtp_gemm_skinny.  The workspace (device, 16-byte aligned, at least
  * ptqtp_gemm_skinny_workspace_size(shape, m) bytes, contents irrelevant on entry, clobbered on return) holds X

@@ -22,7 +22,7 @@ MAX_BATCH = 64
 OK, ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_SIZE, ERR_TRIT, ERR_FORMAT, ERR_CUDA, ERR_CONFIG = (
     0, -1, -2, -3, -4, -5, -6, -7, -8)
 
-EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny",
+EXPORTS = ("ptqtp_packed_size", "ptqtp_pack", "ptqtp_unpack", "ptqtp_gemv", "ptqtp_gemm_skinny", "ptqtp_gemm_skinny_cfg",
            "ptqtp_gemv_host", "ptqtp_gemv_cfg", "ptqtp_parse_header", "ptqtp_status_string",
            "ptqtp_last_cuda_error", "ptqtp_version", "ptqtp_set_overlap", "ptqtp_gemm_skinny_workspace_size", "ptqtp_gemm_skinny_ws",
            "ptqtp_gemm_skinny_static", "ptqtp_kernel_status", "ptqtp_gemv_swiglu", "ptqtp_kernel_status_clear",
@@ -80,6 +80,8 @@ def lib():
         L.ptqtp_gemv_multi.argtypes = [i32, sp, ctypes.POINTER(vp), ctypes.POINTER(sz), vp, ctypes.POINTER(vp), i32, vp]
         L.ptqtp_gemm_skinny.restype = ctypes.c_int
         L.ptqtp_gemm_skinny.argtypes = [sp, vp, sz, i32, vp, vp, vp]
+        L.ptqtp_gemm_skinny_cfg.restype = ctypes.c_int
+        L.ptqtp_gemm_skinny_cfg.argtypes = [sp, vp, sz, i32, vp, vp, i32, i32, vp]
         L.ptqtp_gemm_skinny_workspace_size.restype = sz
         L.ptqtp_gemm_skinny_workspace_size.argtypes = [sp, i32]
         L.ptqtp_gemm_skinny_ws.restype = ctypes.c_int
@@ -277,6 +279,19 @@ def ptqtp_gemm_skinny(packed, N, K, X, Y=None, stream=None, fmt=None):
                                  int(M), _dev(X, torch.float16, "X"), _dev(Y, torch.float16, "Y"),
                                  _stream_ptr(stream))
     _check(st, "ptqtp_gemm_skinny")
+    return Y
+
+
+def ptqtp_gemm_skinny_cfg(packed, N, K, X, Y=None, path=0, k_split=0, stream=None):
+    """ptqtp_gemm_skinny on format 3 with the kernel chosen by the caller (path 0 / 5 / 6, k_split 0 / 1 / 2 / 4 / 8)."""
+    shape = make_shape(N, K, fmt=FORMAT_V3)
+    M = X.shape[0]
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=X.device)
+    st = lib().ptqtp_gemm_skinny_cfg(ctypes.byref(shape), _dev(packed, torch.uint8, "packed"), packed.numel(),
+                                     int(M), _dev(X, torch.float16, "X"), _dev(Y, torch.float16, "Y"), int(path),
+                                     int(k_split), _stream_ptr(stream))
+    _check(st, "ptqtp_gemm_skinny_cfg")
     return Y
 
 

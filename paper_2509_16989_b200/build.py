@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libptqtp.so")
-SOURCES = ["api.cu", "pack.cu", "pack2.cu", "gemv.cu", "gemv2.cu", "gemv3.cu", "pack3.cu", "gemv4.cu", "gemv5.cu", "skinny3.cu", "decompose.cu"]
+SOURCES = ["api.cu", "pack.cu", "pack2.cu", "gemv.cu", "gemv2.cu", "gemv3.cu", "pack3.cu", "gemv4.cu", "gemv5.cu", "gemm6.cu", "skinny3.cu", "decompose.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--shared", "-cudart", "shared"]
 

@@ -247,6 +247,29 @@ ptqtp_status ptqtp_gemv_multi(int32_t count, const ptqtp_shape* shapes, const vo
     return launch_gemv4_jobs(J, x, 0, 0, 0, 0, static_cast<cudaStream_t>(stream), pair ? 2 : 0);
 }
 
+// Small batch on format 3.  path 6 (the library's choice from kSkinnyTc3 rows on): the tcgen05 kernel, all rows in one
+// pass over the planes.  path 5: up to four rows per pass on the warp-MMA kernel whose MMA columns are the rows (two
+// rows cost about a batch-1 pass, four about one and a half); when four rows of x leave no room in shared memory its
+// passes take two rows, or one on the batch-1 kernel.
+constexpr int kSkinnyTc3 = 5;
+static ptqtp_status skinny_v3(const Layout3& L3, const ptqtp_shape* shape, const void* packed, int m, const uint16_t* X,
+                              uint16_t* Y, int path, int k_split, cudaStream_t st) {
+    if (path == 6 || (path == 0 && m >= kSkinnyTc3)) return launch_gemm6(L3, packed, m, X, Y, k_split, st);
+    int per_pass = m < 4 ? m : 4;
+    int done = 0;
+    while (done < m) {
+        const uint16_t* Xp = X + (size_t)done * shape->k_in;
+        uint16_t* Yp = Y + (size_t)done * shape->n_out;
+        const int rows = m - done < per_pass ? m - done : per_pass;
+        ptqtp_status sp = rows == 1 ? launch_gemv4(L3, packed, Xp, Yp, 0, 0, 0, 0, st)
+                                    : launch_gemv5(L3, packed, rows, Xp, Yp, 0, 0, st);
+        if (sp == PTQTP_ERR_SHAPE && rows > 1 && done == 0) { per_pass = per_pass > 2 ? 2 : 1; continue; }   // nothing launched yet
+        if (sp != PTQTP_OK) return sp;
+        done += rows;
+    }
+    return PTQTP_OK;
+}
+
 ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, int32_t m,
                                const uint16_t* X, uint16_t* Y, void* stream) {
     if (!X || !Y) return PTQTP_ERR_NULL;
@@ -277,27 +300,22 @@ ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape* shape, const void* packed, siz
         }
         return launch_gemv2(L.l2, packed, X, Y, 0, 0, 0, 0, st);
     }
-    if (L.v3) {
-        // Format 3: up to four rows per pass over the planes on the tensor-core kernel whose MMA columns are the rows
-        // (two rows cost about a batch-1 pass, four about one and a half); more rows take a pass per four, and when
-        // four rows of x leave no room in shared memory the passes take two rows, or one on the batch-1 kernel.
-        int per_pass = m < 4 ? m : 4;
-        int done = 0;
-        while (done < m) {
-            const uint16_t* Xp = X + (size_t)done * shape->k_in;
-            uint16_t* Yp = Y + (size_t)done * shape->n_out;
-            const int rows = m - done < per_pass ? m - done : per_pass;
-            ptqtp_status sp = rows == 1 ? launch_gemv4(L.l3, packed, Xp, Yp, 0, 0, 0, 0, st)
-                                        : launch_gemv5(L.l3, packed, rows, Xp, Yp, 0, 0, st);
-            if (sp == PTQTP_ERR_SHAPE && rows > 1 && done == 0) { per_pass = per_pass > 2 ? 2 : 1; continue; }   // nothing launched yet
-            if (sp != PTQTP_OK) return sp;
-            done += rows;
-        }
-        return PTQTP_OK;
-    }
+    if (L.v3) return skinny_v3(L.l3, shape, packed, m, X, Y, 0, 0, st);
     // format 1 is a batch-1 layout
     if (m != 1) return PTQTP_ERR_CONFIG;
     return gemv_any(L, packed, X, Y, 0, 0, 0, 0, -1, st);
+}
+
+ptqtp_status ptqtp_gemm_skinny_cfg(const ptqtp_shape* shape, const void* packed, size_t packed_bytes, int32_t m,
+                                   const uint16_t* X, uint16_t* Y, int32_t path, int32_t k_split, void* stream) {
+    if (!X || !Y) return PTQTP_ERR_NULL;
+    AnyLayout L;
+    ptqtp_status s = check_packed(shape, packed, packed_bytes, &L);
+    if (s != PTQTP_OK) return s;
+    if (m < 1 || m > PTQTP_MAX_BATCH) return PTQTP_ERR_SHAPE;
+    if (!L.v3 || (path != 0 && path != 5 && path != 6)) return PTQTP_ERR_CONFIG;
+    if (!aligned16(X) || !aligned16(Y)) return PTQTP_ERR_ALIGN;
+    return skinny_v3(L.l3, shape, packed, m, X, Y, path, k_split, static_cast<cudaStream_t>(stream));
 }
 
 size_t ptqtp_gemm_skinny_workspace_size(const ptqtp_shape* shape, int32_t m) {

@@ -159,6 +159,9 @@ ptqtp_status launch_gemv4(const Layout3& L, const void* packed, const uint16_t* 
 // 2 <= m <= 4 rows on format 3; PTQTP_ERR_SHAPE when (K, m) leaves no room in shared memory
 ptqtp_status launch_gemv5(const Layout3& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, int warps, int depth,
                           cudaStream_t st);
+// 1 <= m <= 64 rows on format 3, tcgen05 kernel; ksplit = CTAs per cluster sharing the columns (0 = library choice)
+ptqtp_status launch_gemm6(const Layout3& L, const void* packed, int m, const uint16_t* X, uint16_t* Y, int ksplit,
+                          cudaStream_t st);
 size_t decompose_workspace_bytes(long long rows, int t_max);
 void decompose_offsets(long long rows, int t_max, size_t* delta_off, size_t* err_off, size_t* a1_off, size_t* a2_off,
                        size_t* lam_off);
