@@ -28,20 +28,23 @@ namespace ptqtp {
 
 namespace {
 
-constexpr int kThreads6 = 128;
+constexpr int kRows6 = 128;                            // weight rows (= MMA rows) per CTA
+constexpr int kDecoders6 = 2 * kRows6;                 // decoding threads: one per row and plane
+constexpr int kThreads6 = kDecoders6 + 64;             // + the warp that issues the MMAs + the warp that copies the codes
 constexpr int kBlockTiles6 = 8;                        // tiles per CTA and superblock: 128 weight rows
 constexpr int kStage6 = kBlockTiles6 * kTile3;         // 34816 bytes
 constexpr int kStages6 = 2;
+// A stage in shared memory: the 16-byte lane entries of the block's eight tiles regrouped as [chunk][t][tile][row pair]
+// (a warp of row threads then reads 16 consecutive entries: no bank conflicts), then the tiles' scale quads.
+constexpr int kLaneT6 = 64 * 16;                       // bytes between the entries t and t + 1 of a row pair
+constexpr int kChunk6 = 4 * kLaneT6;                   // bytes between chunks
+constexpr int kStageScales6 = 8 * kChunk6;             // 32768: offset of the scale quads (256 bytes per tile)
 constexpr int kTmemCols6 = 256;                        // D: columns 0 .. 2 NPAD - 1; A: columns 128 .. 255
 constexpr int kACol6 = 128;
-constexpr uint32_t kTritLut6 = 0x003C00BCu;            // byte q of the table = high byte of fp16(q - 1); byte 3 = 0
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -51,16 +54,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int limit) {
-    for (int i = 0; i < limit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// Bulk copy global -> this CTA's shared memory, completion counted in bytes on an mbarrier (no multicast).
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
@@ -72,25 +65,36 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t sel) {
+__device__ __forceinline__ uint32_t prmt2(uint32_t a, uint32_t b, uint32_t sel) {
     uint32_t d;
-    asm("prmt.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(a), "r"(sel));
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
     return d;
 }
-
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr) : "memory");
+
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]));
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr));
+}
+// One lane of a converged warp.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t leader;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(leader));
+    return leader;
+}
+// The loads above complete here; the registers pass through so that no use of them can be scheduled earlier.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&a)[8], uint32_t (&b)[8]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                   "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7])
+                 :: "memory");
 }
 
 // Shared-memory matrix descriptor, K-major, no swizzle: core matrices of 8 rows x 16 bytes (128 contiguous bytes);
@@ -126,8 +130,8 @@ template <int NPAD>
 struct Smem6 {
     static constexpr int x_buf = 16 * NPAD * 16;
     static constexpr int x_off = kStages6 * kStage6;
-    static constexpr int bar_off = x_off + 2 * x_buf;          // mbarriers: one per stage, one for the MMAs; then the
-    static constexpr int total = bar_off + 64;                 // word that receives the tensor-memory address
+    static constexpr int bar_off = x_off + 2 * x_buf;          // six mbarriers, the word that receives the tensor-
+    static constexpr int total = bar_off + 128;                // memory address, the give-up flag
 };
 
 // Queue the copies of activation group gg (columns 128 gg ..) into an activation buffer: chunk kc (8 columns) of
@@ -135,33 +139,101 @@ struct Smem6 {
 template <int NPAD>
 __device__ __forceinline__ void fetch_x(const __half* __restrict__ X, int k, int m, int gg, uint32_t buf) {
 #pragma unroll
-    for (int q0 = 0; q0 < 16 * NPAD; q0 += kThreads6) {
+    for (int q0 = 0; q0 < 16 * NPAD; q0 += kDecoders6) {
         const int q = q0 + (int)threadIdx.x;
         const int n = (q >> 1) % NPAD, kc = 2 * ((q >> 1) / NPAD) + (q & 1);
         if (n < m) cp_async16(buf + kc * (NPAD * 16) + n * 16, X + (size_t)n * k + 128 * gg + 8 * kc);
     }
 }
 
+// Wait for a phase of an mbarrier; gives up after `limit` polls or when another thread of the CTA has given up.
+__device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, int limit, volatile int* failed) {
+    for (int i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 31) == 31 && *failed) return false;
+    }
+    *failed = 1;
+    return false;
+}
+
+// Half of the 128 columns of one scale group of this thread's row, both planes: the four 16-column chunks c = 2 cq + hc
+// as fp16 trits into tensor memory (8 columns per chunk and plane).  The row's code sits at the same two bits of
+// every byte (mask0 for plane 0, two bits higher for plane 1); the byte permute puts two code bytes under the
+// exponent of 1024 (0x64 high bytes), so a half holds 1024 + code * 2^s exactly, and one fp16 FMA maps it to
+// code - 1.  The masks and permutes run on the integer pipe, the FMAs on the fp16 pipe.  H: which half of a lane
+// entry holds the group (groups 0, 1 of a superblock: words 0 and 2; groups 2, 3: words 1 and 3).
+template <int H>
+__device__ __forceinline__ void decode_half_group(const unsigned char* lane_entry, int hc, uint32_t mask0, __half2 scale0,
+                                                  __half2 bias0, __half2 scale1, __half2 bias1, uint32_t a_cols) {
+    const uint32_t mask1 = mask0 << 2;
+    // all eight 16-byte loads first: their latencies overlap, the arithmetic follows
+    uint4 v[4][2];
+#pragma unroll
+    for (int cq = 0; cq < 4; ++cq)
+#pragma unroll
+        for (int tt = 0; tt < 2; ++tt)
+            v[cq][tt] = *reinterpret_cast<const uint4*>(lane_entry + (2 * cq + hc) * kChunk6 + tt * kLaneT6);
+#pragma unroll
+    for (int cq = 0; cq < 4; ++cq) {
+        const int c = 2 * cq + hc;
+        uint32_t r0[8], r1[8];
+#pragma unroll
+        for (int tt = 0; tt < 2; ++tt) {
+            const uint32_t w[2] = {H ? v[cq][tt].y : v[cq][tt].x, H ? v[cq][tt].w : v[cq][tt].z};
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                const int col = 4 * s + 2 * tt;                 // columns 8 s + 4 tt .. + 3 of the chunk: two 32-bit columns
+                const uint32_t c0 = w[s] & mask0, c1 = w[s] & mask1;
+                const uint32_t lo0 = prmt2(c0, 0x64646464u, 0x4140u), hi0 = prmt2(c0, 0x64646464u, 0x4342u);
+                const uint32_t lo1 = prmt2(c1, 0x64646464u, 0x4140u), hi1 = prmt2(c1, 0x64646464u, 0x4342u);
+                const __half2 a0 = __hfma2(*reinterpret_cast<const __half2*>(&lo0), scale0, bias0);
+                const __half2 b0 = __hfma2(*reinterpret_cast<const __half2*>(&hi0), scale0, bias0);
+                const __half2 a1 = __hfma2(*reinterpret_cast<const __half2*>(&lo1), scale1, bias1);
+                const __half2 b1 = __hfma2(*reinterpret_cast<const __half2*>(&hi1), scale1, bias1);
+                r0[col] = *reinterpret_cast<const uint32_t*>(&a0);
+                r0[col + 1] = *reinterpret_cast<const uint32_t*>(&b0);
+                r1[col] = *reinterpret_cast<const uint32_t*>(&a1);
+                r1[col + 1] = *reinterpret_cast<const uint32_t*>(&b1);
+            }
+        }
+        tmem_st8(a_cols + 8 * c, r0);
+        tmem_st8(a_cols + 64 + 8 * c, r1);
+    }
+}
+
+// Warps 0-7: two threads per weight row; each decodes half of a group's columns (both planes), reads half of the
+// accumulator columns in the scale epilogue and fetches its share of the activations.  Warp 8 issues the MMAs (the
+// whole warp runs the loop so that the operands stay in uniform registers; one elected lane issues).  Warp 9 keeps
+// the ring of code stages full.  They meet on mbarriers only:
+//   code_full[s]  (32 arrivals)  stage s holds the block's tiles of a superblock (one arrival per copying lane)
+//   code_free[s]  (256 arrivals) every decoder is done with stage s
+//   a_full        (256 arrivals) the group's trits are in tensor memory, its activations in shared memory, and the
+//                                accumulators of the group before have been read
+//   a_free        (MMA commit)   the group's 16 MMAs are done
+// A CTA alternates between decoding and multiplying; the two CTAs of an SM fill each other's gaps.
 template <int NPAD>
 __global__ void __launch_bounds__(kThreads6, 2)
 gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* __restrict__ X, __half* __restrict__ Y,
              int m, int csize, int spin_limit, int inject, int* status_word) {
     extern __shared__ __align__(128) unsigned char smem[];
     using SM = Smem6<NPAD>;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + SM::bar_off);
-    uint64_t& mma_bar = full_bar[kStages6];
-    uint32_t& tmem_slot = *reinterpret_cast<uint32_t*>(full_bar + kStages6 + 1);
+    constexpr int HALF = NPAD / 2;                       // accumulator columns per decoder of a row
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::bar_off);
+    const uint32_t code_full = smem_u32(bars), code_free = smem_u32(bars + 2), a_full = smem_u32(bars + 4),
+                   a_free = smem_u32(bars + 5);
+    uint32_t& tmem_slot = *reinterpret_cast<uint32_t*>(bars + 6);
+    volatile int* failed = reinterpret_cast<volatile int*>(bars + 7);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int crank = (int)blockIdx.x % csize, blk = (int)blockIdx.x / csize;
     const int rb0 = blk * kBlockTiles6;
     const int tiles = min(kBlockTiles6, L.nrb - rb0);
-    const uint32_t stage_bytes = (uint32_t)tiles * kTile3;
     const int groups = L.k / 128;
     // this CTA's superblocks: a balanced split of the superblocks over the cluster
     const int sb_base = L.sbs / csize, sb_rem = L.sbs % csize;
     const int sb_lo = crank * sb_base + min(crank, sb_rem);
     const int sb_hi = sb_lo + sb_base + (crank < sb_rem ? 1 : 0);
+    const int gg_lo = 4 * sb_lo, gg_end = min(4 * sb_hi, groups);
     const unsigned char* codes = packed + L.codes_off;
 
     if (warp == 0) {
@@ -170,8 +242,13 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid == 0) {
-        for (int s = 0; s < kStages6; ++s) mbar_init(&full_bar[s], 1);
-        mbar_init(&mma_bar, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bars + s, 32);
+            mbar_init(bars + 2 + s, kDecoders6);
+        }
+        mbar_init(bars + 4, kDecoders6);
+        mbar_init(bars + 5, 1);
+        *failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // rows m .. NPAD - 1 of the activation buffers stay zero
@@ -181,147 +258,143 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = tmem_slot;
-    const uint32_t tlane = tbase + ((uint32_t)(warp * 32) << 16);       // this warp's 32 lanes
     const uint32_t xbuf0 = smem_u32(smem + SM::x_off);
 
-    if (tid == 0) {
-        for (int s = 0; s < kStages6 && sb_lo + s < sb_hi; ++s) {
-            mbar_expect_tx(smem_u32(&full_bar[s]), stage_bytes);
-            bulk_copy_g2s(smem_u32(smem + s * kStage6), codes + tile_offset3(L, rb0, sb_lo + s), stage_bytes,
-                          smem_u32(&full_bar[s]));
-        }
-    }
-    int gg = 4 * sb_lo;                                  // global group index of the pass at hand
-    const int gg_end = min(4 * sb_hi, groups);
-    if (gg < gg_end) fetch_x<NPAD>(X, L.k, m, gg, xbuf0);
-    cp_async_commit();
+    float y[HALF];
+#pragma unroll
+    for (int i = 0; i < HALF; ++i) y[i] = 0.f;
+    const int hc = (warp >> 2) & 1, row_in = 32 * (warp & 3) + lane;        // decoders only
 
-    // thread -> (tile of the block, row pair g of the tile, member of the pair)
-    const int tl = 2 * warp + (lane >> 4), g = (lane >> 1) & 7, mem = lane & 1;
-    const uint32_t sh = 4u - 4u * (uint32_t)mem;         // brings the row's plane-1 code to bits 4-5 of each byte
-    const uint32_t idesc = (1u << 4) | ((uint32_t)(NPAD >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-
-    float y[NPAD];
-#pragma unroll
-    for (int i = 0; i < NPAD; ++i) y[i] = 0.f;
-    bool failed = false;
-    int pass = 0;
-
-    for (; gg < gg_end; ++gg, ++pass) {
-        const int sb = gg >> 2, G = gg & 3, sl = sb - sb_lo, stage = sl % kStages6;
-        const unsigned char* tile = smem + stage * kStage6 + tl * kTile3;
-        if (G == 0) {
-            const bool ok = !(inject && pass == 0) &&
-                            mbar_wait_bounded(smem_u32(&full_bar[stage]), (uint32_t)(sl / kStages6) & 1u, spin_limit);
-            if (!__syncthreads_and(ok)) { failed = true; break; }
-        }
-        // (1) the next group's activations into the other buffer (its last reader, the MMAs two passes back, is done)
-        if (gg + 1 < gg_end) fetch_x<NPAD>(X, L.k, m, gg + 1, xbuf0 + ((pass + 1) & 1) * SM::x_buf);
-        cp_async_commit();
-
-        // (2) decode this row's 128 columns of both planes into tensor memory
-        const int u = G & 1, h = G >> 1;
-        const __half2 alpha = *reinterpret_cast<const __half2*>(tile + kTileCodes3 + 8 * (4 * g + G) + 4 * mem);
-        // (tiles past the matrix hold whatever the stage held: the lookup yields finite values for any bits, such a
-        // row only feeds its own accumulator lane and is never stored; the stores are warp-wide instructions)
-        {
-#pragma unroll
-            for (int o = 0; o < 4; ++o) {
-                uint32_t r1[16], r2[16];
-#pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-#pragma unroll
-                    for (int tt = 0; tt < 2; ++tt) {
-                        const uint4 v = *reinterpret_cast<const uint4*>(tile + (2 * o + cc) * 512 + (4 * g + 2 * u + tt) * 16);
-                        const uint32_t w[2] = {h ? v.y : v.x, h ? v.w : v.z};
-#pragma unroll
-                        for (int s = 0; s < 2; ++s) {
-                            const uint32_t c = w[s] << sh;
-                            const uint32_t s1 = (c & 0x30303030u) | 0x03030303u;
-                            const uint32_t s2 = ((c >> 2) & 0x30303030u) | 0x03030303u;
-                            const int wq = 4 * cc + 2 * s + tt;             // word of the octet: columns 4 wq .. 4 wq + 3
-                            r1[2 * wq] = prmt(kTritLut6, s1);
-                            r1[2 * wq + 1] = prmt(kTritLut6, s1 >> 16);
-                            r2[2 * wq] = prmt(kTritLut6, s2);
-                            r2[2 * wq + 1] = prmt(kTritLut6, s2 >> 16);
-                        }
-                    }
-                }
-                tmem_st16(tlane + kACol6 + 16 * o, r1);
-                tmem_st16(tlane + kACol6 + 64 + 16 * o, r2);
+    if (warp == 9) {
+        // ---- the ring of code stages: 16-byte asynchronous copies that regroup the lane entries ----
+        bool ok = true;
+        for (int sb = sb_lo; sb < sb_hi && ok; ++sb) {
+            const int sl = sb - sb_lo, stage = sl & 1;
+            if (sl >= kStages6) ok = wait_phase(code_free + 8 * stage, (uint32_t)((sl >> 1) - 1) & 1u, spin_limit, failed);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const unsigned char* src = codes + tile_offset3(L, rb0, sb);
+            const uint32_t dst = smem_u32(smem + stage * kStage6);
+            for (int q = lane; q < tiles * (kTile3 / 16); q += 32) {
+                const int tile = q / (kTile3 / 16), r = q - tile * (kTile3 / 16);
+                const uint32_t off = r < 256 ? (uint32_t)((((r >> 5) * 4 + (r & 3)) * 64 + tile * 8 + ((r >> 2) & 7)) * 16)
+                                             : (uint32_t)(kStageScales6 + tile * 256 + (r - 256) * 16);
+                cp_async16(dst + off, src + (size_t)q * 16);
             }
+            // the stage's mbarrier counts one arrival per lane, made when the lane's copies have landed
+            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(code_full + 8 * stage) : "memory");
         }
-        // (3) activations of this group landed; operands visible to the tensor core
-        cp_async_wait_all_but_one();
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        tc_fence_before();
-        __syncthreads();
-        // (4) one thread issues the MMAs; the stage is free once the last group of its superblock is decoded
-        if (tid == 0) {
+        cp_async_wait_all();
+    } else if (warp == 8) {
+        // ---- the MMAs ----
+        const uint32_t idesc = (1u << 4) | ((uint32_t)(NPAD >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        const uint32_t leader = elect_one();
+        for (int gg = gg_lo, pass = 0; gg < gg_end; ++gg, ++pass) {
+            const uint64_t bdesc = smem_desc(xbuf0 + (pass & 1) * SM::x_buf, NPAD * 16, 128);
+            const bool ok = wait_phase(a_full, (uint32_t)pass & 1u, spin_limit, failed);
+            if (!__all_sync(0xffffffffu, ok)) break;
             tc_fence_after();
-            const uint32_t xb = xbuf0 + (pass & 1) * SM::x_buf;
+            if (leader) {
 #pragma unroll
-            for (int p = 0; p < 2; ++p)
+                for (int p = 0; p < 2; ++p)
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    mma_f16_ts(tbase + p * NPAD, tbase + kACol6 + 64 * p + 8 * j,
-                               smem_desc(xb + 2 * j * (NPAD * 16), NPAD * 16, 128), idesc, j > 0 ? 1u : 0u);
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                         ::"r"(smem_u32(&mma_bar)) : "memory");
-            if ((G == 3 || gg + 1 == gg_end) && sb + kStages6 < sb_hi) {
-                mbar_expect_tx(smem_u32(&full_bar[stage]), stage_bytes);
-                bulk_copy_g2s(smem_u32(smem + stage * kStage6), codes + tile_offset3(L, rb0, sb + kStages6), stage_bytes,
-                              smem_u32(&full_bar[stage]));
+                    for (int j = 0; j < 8; ++j)        // a k-step further on: two chunks of NPAD * 16 bytes
+                        mma_f16_ts(tbase + p * NPAD, tbase + kACol6 + 64 * p + 8 * j, bdesc + (uint64_t)(2 * j * NPAD),
+                                   idesc, j > 0 ? 1u : 0u);
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                             ::"r"(a_free) : "memory");
             }
+            __syncwarp();
         }
-        // (5) wait for the MMAs, (6) scale epilogue
-        {
-            const bool ok = mbar_wait_bounded(smem_u32(&mma_bar), (uint32_t)pass & 1u, spin_limit);
-            if (!__syncthreads_and(ok)) { failed = true; break; }
-        }
-        tc_fence_after();
-        const float a1 = __low2float(alpha), a2 = __high2float(alpha);
-#pragma unroll
-        for (int c0 = 0; c0 < NPAD; c0 += 16) {
-            uint32_t d1[16], d2[16];
-            tmem_ld16(tlane + c0, d1);
-            tmem_ld16(tlane + NPAD + c0, d2);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-            for (int i = 0; i < 16; ++i)
-                y[c0 + i] = fmaf(a1, __uint_as_float(d1[i]), fmaf(a2, __uint_as_float(d2[i]), y[c0 + i]));
-        }
-        tc_fence_before();
-    }
-    cp_async_wait_all();
+    } else {
+        // ---- two threads per weight row ----
+        const uint32_t tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);      // this warp's 32 lanes
+        // thread -> (tile of the block, row pair g of the tile, member of the pair)
+        const int tl = row_in >> 4, g = (lane >> 1) & 7, mem = lane & 1;
+        // the row's codes: plane 0 at bits 4 mem .. 4 mem + 1 of every byte, plane 1 two bits higher
+        const uint32_t mask0 = 0x03030303u << (4 * mem);
+        const __half2 scale0 = __float2half2_rn(mem ? 0.0625f : 1.f), bias0 = __float2half2_rn(mem ? -65.f : -1025.f);
+        const __half2 scale1 = __float2half2_rn(mem ? 0.015625f : 0.25f), bias1 = __float2half2_rn(mem ? -17.f : -257.f);
+        bool ok = true;
+        __half2 alpha_prev = __float2half2_rn(0.f);
 
-    if (failed) {
+        if (gg_lo < gg_end) fetch_x<NPAD>(X, L.k, m, gg_lo, xbuf0);
+        cp_async_commit();
+        int pass = 0;
+        for (int gg = gg_lo; gg <= gg_end && gg_lo < gg_end; ++gg, ++pass) {
+            const bool live = gg < gg_end;                  // the last round only reads the last group's accumulators
+            const int sb = gg >> 2, G = gg & 3, sl = sb - sb_lo, stage = sl & 1;
+            const unsigned char* stage_base = smem + stage * kStage6;
+            if (pass > 0) {
+                // accumulators of the previous group: y += alpha1 d1 + alpha2 d2 on this thread's half of the columns
+                ok = ok && wait_phase(a_free, (uint32_t)(pass - 1) & 1u, spin_limit, failed);
+                if (!__all_sync(0xffffffffu, ok)) { *failed = 1; break; }
+                tc_fence_after();
+                const float a1 = __low2float(alpha_prev), a2 = __high2float(alpha_prev);
+#pragma unroll
+                for (int c0 = 0; c0 < HALF; c0 += 8) {
+                    uint32_t d1[8], d2[8];
+                    tmem_ld8(tlane + hc * HALF + c0, d1);
+                    tmem_ld8(tlane + NPAD + hc * HALF + c0, d2);
+                    tmem_ld_wait(d1, d2);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        y[c0 + i] = fmaf(a1, __uint_as_float(d1[i]), fmaf(a2, __uint_as_float(d2[i]), y[c0 + i]));
+                }
+                tc_fence_before();
+            }
+            if (!live) break;
+            // the buffer of the group after this one was last read by the MMAs of the previous group: done
+            if (gg + 1 < gg_end) fetch_x<NPAD>(X, L.k, m, gg + 1, xbuf0 + ((pass + 1) & 1) * SM::x_buf);
+            cp_async_commit();
+            if (G == 0) {
+                ok = !(inject && pass == 0) && wait_phase(code_full + 8 * stage, (uint32_t)(sl >> 1) & 1u, spin_limit, failed);
+                if (!__all_sync(0xffffffffu, ok)) { *failed = 1; break; }
+            }
+            alpha_prev = *reinterpret_cast<const __half2*>(stage_base + kStageScales6 + tl * 256 + 8 * (4 * g + G) + 4 * mem);
+            const unsigned char* lane_entry = stage_base + 2 * (G & 1) * kLaneT6 + (tl * 8 + g) * 16;
+            if (G >> 1) decode_half_group<1>(lane_entry, hc, mask0, scale0, bias0, scale1, bias1, tlane + kACol6);
+            else decode_half_group<0>(lane_entry, hc, mask0, scale0, bias0, scale1, bias1, tlane + kACol6);
+            cp_async_wait_all_but_one();                    // this group's activations (queued one round ago)
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            mbar_arrive(a_full);
+            if (G == 3 || gg + 1 == gg_end) mbar_arrive(code_free + 8 * stage);
+        }
+        cp_async_wait_all();
+    }
+    __syncthreads();
+    const bool bad = *failed != 0;
+    if (bad) {
         if (tid == 0) atomicExch(status_word, (int)PTQTP_ERR_CUDA);
-        // a copy whose wait gave up may still be in flight: give it time to land before the memory is reused
+        // copies and MMAs whose waits gave up may still be in flight: give them time before the memory is reused
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
 #pragma unroll
-        for (int i = 0; i < NPAD; ++i) y[i] = __int_as_float(0x7fc00000);
+        for (int i = 0; i < HALF; ++i) y[i] = __int_as_float(0x7fc00000);
     }
-    const int row = 16 * rb0 + tid;
+    const int row = 16 * rb0 + row_in;
     if (csize == 1) {
-        if (row < L.n) {
+        if (tid < kDecoders6 && row < L.n) {
 #pragma unroll
-            for (int i = 0; i < NPAD; ++i)
-                if (i < m) Y[(size_t)i * L.n + row] = __float2half_rn(y[i]);
+            for (int i = 0; i < HALF; ++i)
+                if (hc * HALF + i < m) Y[(size_t)(hc * HALF + i) * L.n + row] = __float2half_rn(y[i]);
         }
     } else {
         // partial sums of the cluster meet in shared memory; rank r adds its share of the columns in rank order
-        __syncthreads();
         float* P = reinterpret_cast<float*>(smem);
+        if (tid < kDecoders6) {
 #pragma unroll
-        for (int i = 0; i < NPAD; ++i) P[i * kThreads6 + tid] = y[i];
+            for (int i = 0; i < HALF; ++i) P[(hc * HALF + i) * kRows6 + row_in] = y[i];
+        }
         cluster_sync_all();
-        const int per = NPAD / csize;
-        for (int i = crank * per; i < (crank + 1) * per && i < m; ++i) {
-            float s = 0.f;
-            for (int r = 0; r < csize; ++r) s += ld_cluster_f32(smem_u32(P + i * kThreads6 + tid), (uint32_t)r);
-            if (row < L.n) Y[(size_t)i * L.n + row] = __float2half_rn(s);
+        if (tid < kDecoders6) {
+            const int per = NPAD / csize;
+            for (int i = crank * per + hc; i < (crank + 1) * per && i < m; i += 2) {
+                float s = 0.f;
+                for (int r = 0; r < csize; ++r) s += ld_cluster_f32(smem_u32(P + i * kRows6 + row_in), (uint32_t)r);
+                if (row < L.n) Y[(size_t)i * L.n + row] = __float2half_rn(s);
+            }
         }
         cluster_sync_all();
     }
