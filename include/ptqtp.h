@@ -194,11 +194,16 @@ PTQTP_API ptqtp_status ptqtp_gemv_multi(int32_t count, const ptqtp_shape *shapes
  * one pass over the planes at about the cost of a batch-1 call (the activations stay in registers); larger M
  * take one such pass per four rows (ptqtp_gemm_skinny_ws reads the planes once for any M).  When four rows of x
  * leave no room in shared memory (very long K) the passes take three or two rows, or one row on the batch-1
- * kernel.  M = 1 runs the batch-1 kernel.  Format 3: the same tiles and decode as its batch-1 kernel, with the MMA
- * columns holding two or four batch rows instead of the four scale groups (two or four times the tensor-core work
- * of one row, the same masks and the same stream of tiles); M = 2 takes one pass at about 1.3 times the cost of a
- * batch-1 call, larger M take a pass per four rows (two when four rows of x leave no room in shared memory); format
- * 2 is the faster small-batch layout from M = 3 on.  Format 1 is a batch-1 layout: M > 1 returns PTQTP_ERR_CONFIG. */
+ * kernel.  M = 1 runs the batch-1 kernel.  Format 3, few rows: the same tiles and decode as its batch-1 kernel, with
+ * the MMA columns holding two or four batch rows instead of the four scale groups (two or four times the
+ * tensor-core work of one row, the same masks and the same stream of tiles); M = 2 takes one pass at about 1.3
+ * times the cost of a batch-1 call, larger M take a pass per four rows (two when four rows of x leave no room in
+ * shared memory).  Format 3, more rows (from M = 5 to about 20, later for small matrices: the library compares the
+ * measured costs of both): one pass over the planes for all rows on the tcgen05 tensor cores -- the codes
+ * are decoded to fp16 trits in tensor memory (the A operand), the activations are the fp16 B operand as given (no
+ * quantisation), the sums of a scale group accumulate in fp32 in tensor memory and get the fp32 scale epilogue;
+ * matrices with few rows split K over a thread-block cluster and add the partial sums in rank order
+ * (reproducible).  Format 1 is a batch-1 layout: M > 1 returns PTQTP_ERR_CONFIG. */
 PTQTP_API ptqtp_status ptqtp_gemm_skinny(const ptqtp_shape *shape /* host */, const void *packed,
                                size_t packed_bytes, int32_t m, const uint16_t *X, uint16_t *Y,
                                void *stream);

@@ -247,14 +247,24 @@ ptqtp_status ptqtp_gemv_multi(int32_t count, const ptqtp_shape* shapes, const vo
     return launch_gemv4_jobs(J, x, 0, 0, 0, 0, static_cast<cudaStream_t>(stream), pair ? 2 : 0);
 }
 
-// Small batch on format 3.  path 6 (the library's choice from kSkinnyTc3 rows on): the tcgen05 kernel, all rows in one
-// pass over the planes.  path 5: up to four rows per pass on the warp-MMA kernel whose MMA columns are the rows (two
-// rows cost about a batch-1 pass, four about one and a half); when four rows of x leave no room in shared memory its
-// passes take two rows, or one on the batch-1 kernel.
-constexpr int kSkinnyTc3 = 5;
+// Small batch on format 3.  path 5: up to four rows per pass over the planes on the warp-MMA kernel whose MMA columns
+// are the rows (two rows cost about a batch-1 pass, four about one and a half); when four rows of x leave no room in
+// shared memory its passes take two rows, or one on the batch-1 kernel.  path 6: the tcgen05 kernel, all rows in one
+// pass.  path 0: whichever the measured costs below make cheaper -- the tcgen05 kernel has a fixed cost of several
+// microseconds and a cost per byte that grows slowly with the rows, the passes cost a batch-1 call each.
+static bool tcgen05_is_cheaper(const Layout3& L3, int m) {
+    if (m < 5) return false;
+    const double mb = (double)L3.total / 1e6;
+    const int npad = (m + 15) / 16 * 16;
+    const double us6 = 7.5 + mb * (0.52 + 0.015 * npad);
+    const double rate4 = L3.k > 8192 ? 1.15 : 2.1, rate2 = 2.0 * rate4;           // MB per microsecond of a pass
+    const int full = m / 4, rest = m % 4;
+    const double us5 = full * (1.2 + mb / rate4) + (rest > 2 ? 1.2 + mb / rate4 : rest > 0 ? 1.2 + mb / rate2 : 0.0);
+    return us6 < us5;
+}
 static ptqtp_status skinny_v3(const Layout3& L3, const ptqtp_shape* shape, const void* packed, int m, const uint16_t* X,
                               uint16_t* Y, int path, int k_split, cudaStream_t st) {
-    if (path == 6 || (path == 0 && m >= kSkinnyTc3)) return launch_gemm6(L3, packed, m, X, Y, k_split, st);
+    if (path == 6 || (path == 0 && tcgen05_is_cheaper(L3, m))) return launch_gemm6(L3, packed, m, X, Y, k_split, st);
     int per_pass = m < 4 ? m : 4;
     int done = 0;
     while (done < m) {

@@ -73,6 +73,12 @@ __device__ __forceinline__ uint32_t prmt2(uint32_t a, uint32_t b, uint32_t sel) 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One arrival for the whole (converged) warp: arrivals on one mbarrier are serialised, 256 of them cost more than
+// the work they separate.  The warp barrier orders every lane's earlier operations before lane 0's release.
+__device__ __forceinline__ void warp_arrive(uint32_t bar) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
 
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
@@ -134,19 +140,31 @@ struct Smem6 {
     static constexpr int total = bar_off + 128;                // memory address, the give-up flag
 };
 
-// Queue the copies of activation group gg (columns 128 gg ..) into an activation buffer: chunk kc (8 columns) of
-// row n goes to kc * NPAD * 16 + n * 16.  Adjacent threads take the two halves of a 32-byte sector.
+// The copies of one activation group (128 columns of every row of X) into an activation buffer: chunk kc (8 columns)
+// of row n goes to kc * NPAD * 16 + n * 16.  A decoder owns NPAD / 16 chunks, the same ones for every group (adjacent
+// threads take the two halves of a 32-byte sector); XChunks holds their offsets.
 template <int NPAD>
-__device__ __forceinline__ void fetch_x(const __half* __restrict__ X, int k, int m, int gg, uint32_t buf) {
+struct XChunks {
+    uint32_t src[NPAD / 16];     // offset in X, in halves, without the group's 128 gg; 0xffffffff: a row past m
+    uint32_t dst[NPAD / 16];     // byte offset in the buffer
+    __device__ __forceinline__ void init(int k, int m) {
 #pragma unroll
-    for (int q0 = 0; q0 < 16 * NPAD; q0 += kDecoders6) {
-        const int q = q0 + (int)threadIdx.x;
-        const int n = (q >> 1) % NPAD, kc = 2 * ((q >> 1) / NPAD) + (q & 1);
-        if (n < m) cp_async16(buf + kc * (NPAD * 16) + n * 16, X + (size_t)n * k + 128 * gg + 8 * kc);
+        for (int i = 0; i < NPAD / 16; ++i) {
+            const int q = i * kDecoders6 + (int)threadIdx.x;
+            const int n = (q >> 1) % NPAD, kc = 2 * ((q >> 1) / NPAD) + (q & 1);
+            src[i] = n < m ? (uint32_t)(n * k + 8 * kc) : 0xffffffffu;
+            dst[i] = (uint32_t)(kc * (NPAD * 16) + n * 16);
+        }
     }
-}
+    __device__ __forceinline__ void fetch(const __half* __restrict__ X, int gg, uint32_t buf) const {
+#pragma unroll
+        for (int i = 0; i < NPAD / 16; ++i)
+            if (src[i] != 0xffffffffu) cp_async16(buf + dst[i], X + src[i] + 128 * gg);
+    }
+};
 
-// Wait for a phase of an mbarrier; gives up after `limit` polls or when another thread of the CTA has given up.
+// Wait for a phase of an mbarrier (the suspending form: a waiting thread takes no issue slots; polling without
+// suspension was measured 30 % slower).  Gives up after `limit` polls or when another thread of the CTA has given up.
 __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, int limit, volatile int* failed) {
     for (int i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -156,26 +174,32 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, int li
     return false;
 }
 
-// Half of the 128 columns of one scale group of this thread's row, both planes: the four 16-column chunks c = 2 cq + hc
-// as fp16 trits into tensor memory (8 columns per chunk and plane).  The row's code sits at the same two bits of
-// every byte (mask0 for plane 0, two bits higher for plane 1); the byte permute puts two code bytes under the
-// exponent of 1024 (0x64 high bytes), so a half holds 1024 + code * 2^s exactly, and one fp16 FMA maps it to
-// code - 1.  The masks and permutes run on the integer pipe, the FMAs on the fp16 pipe.  H: which half of a lane
-// entry holds the group (groups 0, 1 of a superblock: words 0 and 2; groups 2, 3: words 1 and 3).
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    // volatile: stays ahead of the tensor-memory stores that follow in program order, so the loads of a step are
+    // all in flight before the arithmetic on the first of them
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// A quarter of the 128 columns of one scale group of this thread's row, both planes: the two 16-column chunks
+// c = c_first and c_first + 2, as fp16 trits into tensor memory (8 columns per chunk and plane).  The row's code sits
+// at the same two bits of every byte (mask0 for plane 0, two bits higher for plane 1); the byte permute puts two code
+// bytes under the exponent of 1024 (0x64 high bytes), so a half holds 1024 + code * 2^s exactly, and one fp16 FMA
+// maps it to code - 1.  The masks and permutes run on the integer pipe, the FMAs on the fp16 pipe.  H: which half of
+// a lane entry holds the group (groups 0, 1 of a superblock: words 0 and 2; groups 2, 3: words 1 and 3).
 template <int H>
-__device__ __forceinline__ void decode_half_group(const unsigned char* lane_entry, int hc, uint32_t mask0, __half2 scale0,
+__device__ __forceinline__ void decode_two_chunks(uint32_t lane_entry, int c_first, uint32_t mask0, __half2 scale0,
                                                   __half2 bias0, __half2 scale1, __half2 bias1, uint32_t a_cols) {
     const uint32_t mask1 = mask0 << 2;
-    // all eight 16-byte loads first: their latencies overlap, the arithmetic follows
-    uint4 v[4][2];
+    uint4 v[2][2];
 #pragma unroll
-    for (int cq = 0; cq < 4; ++cq)
+    for (int cq = 0; cq < 2; ++cq)
 #pragma unroll
-        for (int tt = 0; tt < 2; ++tt)
-            v[cq][tt] = *reinterpret_cast<const uint4*>(lane_entry + (2 * cq + hc) * kChunk6 + tt * kLaneT6);
+        for (int tt = 0; tt < 2; ++tt) v[cq][tt] = lds128(lane_entry + (c_first + 2 * cq) * kChunk6 + tt * kLaneT6);
 #pragma unroll
-    for (int cq = 0; cq < 4; ++cq) {
-        const int c = 2 * cq + hc;
+    for (int cq = 0; cq < 2; ++cq) {
+        const int c = c_first + 2 * cq;
         uint32_t r0[8], r1[8];
 #pragma unroll
         for (int tt = 0; tt < 2; ++tt) {
@@ -204,13 +228,14 @@ __device__ __forceinline__ void decode_half_group(const unsigned char* lane_entr
 // Warps 0-7: two threads per weight row; each decodes half of a group's columns (both planes), reads half of the
 // accumulator columns in the scale epilogue and fetches its share of the activations.  Warp 8 issues the MMAs (the
 // whole warp runs the loop so that the operands stay in uniform registers; one elected lane issues).  Warp 9 keeps
-// the ring of code stages full.  They meet on mbarriers only:
+// the ring of code stages full.  They meet on mbarriers only (h = 0: k-steps 0-3 of a group, h = 1: k-steps 4-7):
 //   code_full[s]  (32 arrivals)  stage s holds the block's tiles of a superblock (one arrival per copying lane)
-//   code_free[s]  (256 arrivals) every decoder is done with stage s
-//   a_full        (256 arrivals) the group's trits are in tensor memory, its activations in shared memory, and the
-//                                accumulators of the group before have been read
-//   a_free        (MMA commit)   the group's 16 MMAs are done
-// A CTA alternates between decoding and multiplying; the two CTAs of an SM fill each other's gaps.
+//   code_free[s]  (8 arrivals: one per decoding warp) every decoder is done with stage s
+//   a_full[h]     (8 arrivals)   half h of the group's trits is in tensor memory; for h = 0 also: the group's
+//                                activations are in shared memory and the accumulators of the group before are read
+//   a_free[h]     (MMA commit)   the 8 MMAs of half h are done; for h = 1: the group's accumulators are complete
+// The first half of group g + 1 is decoded under the MMAs of the second half of group g, the second half under the
+// MMAs of the first; the two CTAs of an SM fill each other's remaining gaps.
 template <int NPAD>
 __global__ void __launch_bounds__(kThreads6, 2)
 gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* __restrict__ X, __half* __restrict__ Y,
@@ -220,9 +245,9 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
     constexpr int HALF = NPAD / 2;                       // accumulator columns per decoder of a row
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::bar_off);
     const uint32_t code_full = smem_u32(bars), code_free = smem_u32(bars + 2), a_full = smem_u32(bars + 4),
-                   a_free = smem_u32(bars + 5);
-    uint32_t& tmem_slot = *reinterpret_cast<uint32_t*>(bars + 6);
-    volatile int* failed = reinterpret_cast<volatile int*>(bars + 7);
+                   a_free = smem_u32(bars + 6);
+    uint32_t& tmem_slot = *reinterpret_cast<uint32_t*>(bars + 8);
+    volatile int* failed = reinterpret_cast<volatile int*>(bars + 9);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int crank = (int)blockIdx.x % csize, blk = (int)blockIdx.x / csize;
@@ -244,10 +269,12 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
             mbar_init(bars + s, 32);
-            mbar_init(bars + 2 + s, kDecoders6);
+            mbar_init(bars + 2 + s, kDecoders6 / 32);
         }
-        mbar_init(bars + 4, kDecoders6);
-        mbar_init(bars + 5, 1);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(bars + 4 + h, kDecoders6 / 32);
+            mbar_init(bars + 6 + h, 1);
+        }
         *failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -275,11 +302,12 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
             if (!ok) break;
             const unsigned char* src = codes + tile_offset3(L, rb0, sb);
             const uint32_t dst = smem_u32(smem + stage * kStage6);
-            for (int q = lane; q < tiles * (kTile3 / 16); q += 32) {
-                const int tile = q / (kTile3 / 16), r = q - tile * (kTile3 / 16);
-                const uint32_t off = r < 256 ? (uint32_t)((((r >> 5) * 4 + (r & 3)) * 64 + tile * 8 + ((r >> 2) & 7)) * 16)
-                                             : (uint32_t)(kStageScales6 + tile * 256 + (r - 256) * 16);
-                cp_async16(dst + off, src + (size_t)q * 16);
+            for (int tile = 0; tile < tiles; ++tile) {
+                const unsigned char* ts = src + (size_t)tile * kTile3;
+                const uint32_t td = dst + (uint32_t)(((lane & 3) * 64 + tile * 8 + (lane >> 2)) * 16);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) cp_async16(td + c * kChunk6, ts + c * 512 + lane * 16);     // lane entry (c, lane)
+                if (lane < 16) cp_async16(dst + kStageScales6 + tile * 256 + lane * 16, ts + kTileCodes3 + lane * 16);
             }
             // the stage's mbarrier counts one arrival per lane, made when the lane's copies have landed
             asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(code_full + 8 * stage) : "memory");
@@ -289,22 +317,27 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
         // ---- the MMAs ----
         const uint32_t idesc = (1u << 4) | ((uint32_t)(NPAD >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
         const uint32_t leader = elect_one();
-        for (int gg = gg_lo, pass = 0; gg < gg_end; ++gg, ++pass) {
+        bool ok = true;
+        for (int gg = gg_lo, pass = 0; gg < gg_end && ok; ++gg, ++pass) {
             const uint64_t bdesc = smem_desc(xbuf0 + (pass & 1) * SM::x_buf, NPAD * 16, 128);
-            const bool ok = wait_phase(a_full, (uint32_t)pass & 1u, spin_limit, failed);
-            if (!__all_sync(0xffffffffu, ok)) break;
-            tc_fence_after();
-            if (leader) {
 #pragma unroll
-                for (int p = 0; p < 2; ++p)
+            for (int h = 0; h < 2; ++h) {
+                ok = wait_phase(a_full + 8 * h, (uint32_t)pass & 1u, spin_limit, failed);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (leader) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)        // a k-step further on: two chunks of NPAD * 16 bytes
-                        mma_f16_ts(tbase + p * NPAD, tbase + kACol6 + 64 * p + 8 * j, bdesc + (uint64_t)(2 * j * NPAD),
-                                   idesc, j > 0 ? 1u : 0u);
-                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                             ::"r"(a_free) : "memory");
+                    for (int p = 0; p < 2; ++p)
+#pragma unroll
+                        for (int j = 4 * h; j < 4 * h + 4; ++j)     // a k-step further on: two chunks of NPAD * 16 bytes
+                            mma_f16_ts(tbase + p * NPAD, tbase + kACol6 + 64 * p + 8 * j, bdesc + (uint64_t)(2 * j * NPAD),
+                                       idesc, j > 0 ? 1u : 0u);
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                                 ::"r"(a_free + 8 * h) : "memory");
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
     } else {
         // ---- two threads per weight row ----
@@ -318,16 +351,31 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
         bool ok = true;
         __half2 alpha_prev = __float2half2_rn(0.f);
 
-        if (gg_lo < gg_end) fetch_x<NPAD>(X, L.k, m, gg_lo, xbuf0);
+        XChunks<NPAD> xc;
+        xc.init(L.k, m);
+        if (gg_lo < gg_end) xc.fetch(X, gg_lo, xbuf0);
         cp_async_commit();
+        const uint32_t a_cols = tlane + kACol6;
+        __half2 alpha = alpha_prev;
         int pass = 0;
         for (int gg = gg_lo; gg <= gg_end && gg_lo < gg_end; ++gg, ++pass) {
             const bool live = gg < gg_end;                  // the last round only reads the last group's accumulators
             const int sb = gg >> 2, G = gg & 3, sl = sb - sb_lo, stage = sl & 1;
             const unsigned char* stage_base = smem + stage * kStage6;
+            const uint32_t lane_entry = smem_u32(stage_base) + 2 * (G & 1) * kLaneT6 + (tl * 8 + g) * 16;
+            if (live) {
+                // first half of the group's k-steps: under the MMAs of the second half of the group before
+                if (G == 0) ok = ok && !(inject && pass == 0) && wait_phase(code_full + 8 * stage, (uint32_t)(sl >> 1) & 1u, spin_limit, failed);
+                if (pass > 0) ok = ok && wait_phase(a_free, (uint32_t)(pass - 1) & 1u, spin_limit, failed);
+                if (!__all_sync(0xffffffffu, ok)) { *failed = 1; break; }
+                tc_fence_after();
+                alpha = *reinterpret_cast<const __half2*>(stage_base + kStageScales6 + tl * 256 + 8 * (4 * g + G) + 4 * mem);
+                if (G >> 1) decode_two_chunks<1>(lane_entry, hc, mask0, scale0, bias0, scale1, bias1, a_cols);
+                else decode_two_chunks<0>(lane_entry, hc, mask0, scale0, bias0, scale1, bias1, a_cols);
+            }
             if (pass > 0) {
                 // accumulators of the previous group: y += alpha1 d1 + alpha2 d2 on this thread's half of the columns
-                ok = ok && wait_phase(a_free, (uint32_t)(pass - 1) & 1u, spin_limit, failed);
+                ok = ok && wait_phase(a_free + 8, (uint32_t)(pass - 1) & 1u, spin_limit, failed);
                 if (!__all_sync(0xffffffffu, ok)) { *failed = 1; break; }
                 tc_fence_after();
                 const float a1 = __low2float(alpha_prev), a2 = __high2float(alpha_prev);
@@ -341,26 +389,24 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
                     for (int i = 0; i < 8; ++i)
                         y[c0 + i] = fmaf(a1, __uint_as_float(d1[i]), fmaf(a2, __uint_as_float(d2[i]), y[c0 + i]));
                 }
-                tc_fence_before();
             }
             if (!live) break;
+            alpha_prev = alpha;
             // the buffer of the group after this one was last read by the MMAs of the previous group: done
-            if (gg + 1 < gg_end) fetch_x<NPAD>(X, L.k, m, gg + 1, xbuf0 + ((pass + 1) & 1) * SM::x_buf);
+            if (gg + 1 < gg_end) xc.fetch(X, gg + 1, xbuf0 + ((pass + 1) & 1) * SM::x_buf);
             cp_async_commit();
-            if (G == 0) {
-                ok = !(inject && pass == 0) && wait_phase(code_full + 8 * stage, (uint32_t)(sl >> 1) & 1u, spin_limit, failed);
-                if (!__all_sync(0xffffffffu, ok)) { *failed = 1; break; }
-            }
-            alpha_prev = *reinterpret_cast<const __half2*>(stage_base + kStageScales6 + tl * 256 + 8 * (4 * g + G) + 4 * mem);
-            const unsigned char* lane_entry = stage_base + 2 * (G & 1) * kLaneT6 + (tl * 8 + g) * 16;
-            if (G >> 1) decode_half_group<1>(lane_entry, hc, mask0, scale0, bias0, scale1, bias1, tlane + kACol6);
-            else decode_half_group<0>(lane_entry, hc, mask0, scale0, bias0, scale1, bias1, tlane + kACol6);
             cp_async_wait_all_but_one();                    // this group's activations (queued one round ago)
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             tc_fence_before();
-            mbar_arrive(a_full);
-            if (G == 3 || gg + 1 == gg_end) mbar_arrive(code_free + 8 * stage);
+            warp_arrive(a_full);
+            // second half: under the MMAs of the first
+            if (G >> 1) decode_two_chunks<1>(lane_entry, 4 + hc, mask0, scale0, bias0, scale1, bias1, a_cols);
+            else decode_two_chunks<0>(lane_entry, 4 + hc, mask0, scale0, bias0, scale1, bias1, a_cols);
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            warp_arrive(a_full + 8);
+            if (G == 3 || gg + 1 == gg_end) warp_arrive(code_free + 8 * stage);
         }
         cp_async_wait_all();
     }

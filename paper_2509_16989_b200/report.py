@@ -3,11 +3,12 @@
     python -m paper_2509_16989_b200.report [--only 0,2,3] [--format 3]
 
 Batch-1 calls use the packed format given by --format (default 3: tiles in int8 MMA operand order; 2: the
-CUDA-core kernel); the small-batch calls (M > 1) always use format 2.  The program opts in to overlap level 2, as
+CUDA-core kernel); the small-batch calls (M > 1) use format 2 unless a line says format 3.  The program opts in to overlap level 2, as
 a decoder would whose packed blobs never change while GEMV calls are in flight.
 
   0  Qwen3-0.6B up_proj 3072 x 1024, batch 1
-  2  batch sweep M in {1,...,64} of ptqtp_gemm_skinny on the 14336 x 4096 gate/up shape (and ptqtp_gemv at M = 1)
+  2  batch sweep M in {1,...,64} of ptqtp_gemm_skinny on the 14336 x 4096 gate/up shape (and ptqtp_gemv at M = 1) on
+     format 2, then M in {2,...,64} on format 3 for the four distinct LLaMA-3-8B shapes
   3  LLaMA-3-70B shapes, planes with P(0) = 0.5, batch 1 and 8
   5  a LLaMA-3-8B layer with stacked matrices: q, k, v packed as one 6144 x 4096 matrix, and also gate, up as one
      28672 x 4096 matrix (rows are independent, so a caller may stack matrices that share their input and
@@ -142,6 +143,25 @@ def config2(T):
                           for b in bufs])
         emit(workload="cfg2 gate/up batch sweep", call="ptqtp_gemm_skinny_ws", N=N, K=K, M=M, us=round(us, 3),
              us_per_batch_row=round(us / M, 3), gbs=round(nb / us / 1e3, 1), bytes=nb)
+    del bufs
+    torch.cuda.empty_cache()
+    # the same sweep on format 3 (M = 2..7: warp-MMA passes of four rows; M >= 8: the tcgen05 kernel), every 8B shape
+    for name in ("gate", "down", "q", "k"):
+        N, K = LLAMA3_8B[name]
+        c = make_case(N, K, seed=2, M=64)
+        packed, st = binding.ptqtp_pack(dev(c["T1"]), dev(c["T2"]), dev(c["alpha1"]), dev(c["alpha2"]), fmt=binding.FORMAT_V3)
+        bufs = T.copies(packed)
+        Xall = dev(c["x"])
+        for M in (2, 4, 8, 16, 32, 64):
+            X = Xall[:M].contiguous()
+            Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+            us = T.steady_us([lambda b=b: binding.ptqtp_gemm_skinny(b, N, K, X, Y=Y, stream=T.stream, fmt=binding.FORMAT_V3)
+                              for b in bufs])
+            nb = algorithmic_bytes(N, K, M)
+            emit(workload="cfg2 format 3 batch sweep " + name, call="ptqtp_gemm_skinny", N=N, K=K, M=M, us=round(us, 3),
+                 us_per_batch_row=round(us / M, 3), gbs=round(nb / us / 1e3, 1), bytes=nb)
+        del bufs
+        torch.cuda.empty_cache()
 
 
 def config3(T):

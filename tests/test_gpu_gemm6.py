@@ -78,21 +78,23 @@ def test_rows_do_not_depend_on_their_neighbours():
     assert np.array_equal(full[8:24].view(np.uint16), part.view(np.uint16))
 
 
-def test_library_dispatch_uses_it_from_five_rows_on():
-    N, K = 520, 3072
-    for M in (5, 16, 64):
-        c = make_case(N, K, seed=40 + M, M=M)
-        packed = pack_case(c, V3)
-        a = binding.ptqtp_gemm_skinny(packed, N, K, dev(c["x"]), fmt=V3)
-        b = binding.ptqtp_gemm_skinny_cfg(packed, N, K, dev(c["x"]), path=6)
+def test_library_dispatch():
+    # the library takes the tcgen05 kernel where its fixed cost pays: many rows, or a matrix of some size
+    def same(a, b):
         torch.cuda.synchronize()
-        assert np.array_equal(a.cpu().numpy().view(np.uint16), b.cpu().numpy().view(np.uint16))
-    c = make_case(N, K, seed=44, M=4)
+        return np.array_equal(a.cpu().numpy().view(np.uint16), b.cpu().numpy().view(np.uint16))
+    N, K = 4096, 4096
+    c = make_case(N, K, seed=40, M=64)
     packed = pack_case(c, V3)
-    a = binding.ptqtp_gemm_skinny(packed, N, K, dev(c["x"]), fmt=V3)
-    b = binding.ptqtp_gemm_skinny_cfg(packed, N, K, dev(c["x"]), path=5)
-    torch.cuda.synchronize()
-    assert np.array_equal(a.cpu().numpy().view(np.uint16), b.cpu().numpy().view(np.uint16))
+    for M, path in ((64, 6), (16, 6), (4, 5)):
+        X = dev(c["x"][:M].copy())
+        assert same(binding.ptqtp_gemm_skinny(packed, N, K, X, fmt=V3), binding.ptqtp_gemm_skinny_cfg(packed, N, K, X, path=path)), M
+    N, K = 520, 3072
+    c = make_case(N, K, seed=41, M=64)
+    packed = pack_case(c, V3)
+    for M, path in ((64, 6), (8, 5), (7, 5)):
+        X = dev(c["x"][:M].copy())
+        assert same(binding.ptqtp_gemm_skinny(packed, N, K, X, fmt=V3), binding.ptqtp_gemm_skinny_cfg(packed, N, K, X, path=path)), M
 
 
 def test_argument_checks():

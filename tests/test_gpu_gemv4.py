@@ -323,7 +323,8 @@ def test_several_matrices_argument_checks():
                                    (64, 14336, 4), (1000, 6144, 7), (37, 36864, 4), (192, 3072, 64), (2400, 4096, 9),
                                    (14336, 4096, 2), (4096, 14336, 4), (1024, 4096, 3), (4096, 4096, 8)])
 def test_small_batch_on_the_batch1_layout(N, K, M, level):
-    # ptqtp_gemm_skinny on format 3: passes of up to four rows on the kernel whose MMA columns are the batch rows
+    # ptqtp_gemm_skinny on format 3: passes of up to four rows on the kernel whose MMA columns are the batch rows, or
+    # (more rows, larger matrices) one pass on the tcgen05 kernel
     binding.ptqtp_set_overlap(level)
     c = make_case(N, K, seed=700 + N + M, M=M)
     packed = pack_case(c, V3)
