@@ -608,6 +608,23 @@ def run_gpu(args):
             detail["step_other_format"] = {"format": other, "kernel": KERNEL_NAME[other],
                                            "us_per_layer": 1e3 * chain.time_ms([go] * 10) / (10 * 4 * R)}
             del go, sets_o, base_o
+            # the small-batch call on the gate/up shape (format 3: warp MMAs for few rows, the tcgen05 kernel for many)
+            if fmt == 3:
+                Ng, Kg = LLAMA3_8B["gate"]
+                small = {}
+                for M in (2, 16, 64):
+                    Xb = torch.randn((M, Kg), generator=torch.Generator(device=device).manual_seed(M), device=device,
+                                     dtype=torch.float32).to(torch.float16)
+                    Yb = torch.empty((M, Ng), dtype=torch.float16, device=device)
+                    call = lambda: [binding.ptqtp_gemm_skinny(sets[r]["gate"], Ng, Kg, Xb, Y=Yb, stream=stream, fmt=3)
+                                    for r in range(R)]
+                    with torch.cuda.stream(stream):
+                        call()
+                        stream.synchronize()
+                    gb = chain.capture(lambda: [call() for _ in range(4)])
+                    small["M%d_us" % M] = 1e3 * chain.time_ms([gb] * 10) / (10 * 4 * R)
+                    del gb
+                detail["small_batch_gate_14336x4096"] = small
 
     sampler.stop()
 
