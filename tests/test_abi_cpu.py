@@ -122,6 +122,16 @@ def test_host_side_validation_codes(L):
             assert L.ptqtp_gemm_skinny(ctypes.byref(sh), ok_ptr, sz, 2, ok_ptr, ok_ptr, None) == binding.ERR_CONFIG
         assert L.ptqtp_gemm_skinny_ws(ctypes.byref(sh), ok_ptr, sz, 2, ok_ptr, ok_ptr, ok_ptr, 1 << 20, None) == binding.ERR_CONFIG
         assert L.ptqtp_gemm_skinny_workspace_size(ctypes.byref(sh), 2) == 0
+    # the kernel choice of the small-batch call exists for format 3 only; paths 0, 5, 6; splits 0, 1, 2, 4, 8
+    s3 = binding.make_shape(8, 256, fmt=binding.FORMAT_V3)
+    z3 = binding.packed_size(8, 256, fmt=binding.FORMAT_V3)
+    assert L.ptqtp_gemm_skinny_cfg(sp, ok_ptr, size, 8, ok_ptr, ok_ptr, 6, 0, None) == binding.ERR_CONFIG
+    assert L.ptqtp_gemm_skinny_cfg(ctypes.byref(s3), ok_ptr, z3, 8, ok_ptr, ok_ptr, 4, 0, None) == binding.ERR_CONFIG
+    assert L.ptqtp_gemm_skinny_cfg(ctypes.byref(s3), ok_ptr, z3, 8, ok_ptr, ok_ptr, 6, 3, None) == binding.ERR_CONFIG
+    assert L.ptqtp_gemm_skinny_cfg(ctypes.byref(s3), ok_ptr, z3, 0, ok_ptr, ok_ptr, 6, 0, None) == binding.ERR_SHAPE
+    assert L.ptqtp_gemm_skinny_cfg(ctypes.byref(s3), ok_ptr, z3, 8, odd_ptr, ok_ptr, 6, 0, None) == binding.ERR_ALIGN
+    assert L.ptqtp_gemm_skinny_cfg(ctypes.byref(s3), ok_ptr, z3, 8, None, ok_ptr, 6, 0, None) == binding.ERR_NULL
+    assert L.ptqtp_gemm_skinny_cfg(ctypes.byref(s3), ok_ptr, z3 - 16, 8, ok_ptr, ok_ptr, 6, 0, None) == binding.ERR_SIZE
 
 
 def test_decompose_host_side_checks(L):
