@@ -392,14 +392,15 @@ gemm6_kernel(Layout3 L, const unsigned char* __restrict__ packed, const __half* 
             }
             if (!live) break;
             alpha_prev = alpha;
-            // the buffer of the group after this one was last read by the MMAs of the previous group: done
-            if (gg + 1 < gg_end) xc.fetch(X, gg + 1, xbuf0 + ((pass + 1) & 1) * SM::x_buf);
-            cp_async_commit();
-            cp_async_wait_all_but_one();                    // this group's activations (queued one round ago)
+            cp_async_wait_all();                            // this group's activations (queued one round ago)
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             tc_fence_before();
             warp_arrive(a_full);
+            // the next group's activations, after the fence (it would wait for copies queued before it): their
+            // buffer was last read by the MMAs of the previous group, which are done
+            if (gg + 1 < gg_end) xc.fetch(X, gg + 1, xbuf0 + ((pass + 1) & 1) * SM::x_buf);
+            cp_async_commit();
             // second half: under the MMAs of the first
             if (G >> 1) decode_two_chunks<1>(lane_entry, 4 + hc, mask0, scale0, bias0, scale1, bias1, a_cols);
             else decode_two_chunks<0>(lane_entry, 4 + hc, mask0, scale0, bias0, scale1, bias1, a_cols);
