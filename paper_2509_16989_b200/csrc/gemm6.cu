@@ -165,7 +165,17 @@ struct XChunks {
 
 // Wait for a phase of an mbarrier (the suspending form: a waiting thread takes no issue slots; polling without
 // suspension was measured 30 % slower).  Gives up after `limit` polls or when another thread of the CTA has given up.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, int limit, volatile int* failed) {
+    if (mbar_test_wait(bar, parity)) return true;        // the usual case: the phase is long complete
     for (int i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 31) == 31 && *failed) return false;
