@@ -404,11 +404,13 @@ def run_gpu(args):
             step(0)
         stream.synchronize()
         worst_rel, worst_frac = 0.0, 0.0
+        refs = {}
         for m in ("q", "k", "gate", "down"):
             c = cases[UNIQUE_OF[m]]
             rows = np.unique(np.random.default_rng(1).integers(0, c["N"], 512))
             ref = layer_fp64_c(c["T1"][rows], c["T2"][rows], c["alpha1"][rows], c["alpha2"][rows], c["x"],
                                threads=max_threads())
+            refs[m] = (rows, ref, c["x"])
             got = ys[m].cpu().numpy()[rows]
             rel, mab, bound = parity_metrics(got, ref, c["x"])[0]
             worst_rel = max(worst_rel, rel)
@@ -421,10 +423,20 @@ def run_gpu(args):
     xh = {m: torch.from_numpy(cases[UNIQUE_OF[m]]["x"].copy()).pin_memory() for m in MATRICES}
     yh = {m: torch.empty(LLAMA3_8B[m][0], dtype=torch.float16).pin_memory() for m in MATRICES}
 
+    # the seven calls of a step are independent of one another (own x, own y): each runs on a stream of its own, forked
+    # from and joined to the step's stream, so their copies and kernels overlap
+    side = [torch.cuda.Stream(device=device) for _ in MATRICES]
+
     def e2e_calls(r):
-        for m in MATRICES:
+        fork = torch.cuda.Event()
+        fork.record(stream)
+        for s_m, m in zip(side, MATRICES):
             N, K = LLAMA3_8B[m]
-            binding.ptqtp_gemv_host(sets[r][m], N, K, xh[m], yh[m], xs[m], ys[m], stream=stream, fmt=fmt)
+            s_m.wait_event(fork)
+            binding.ptqtp_gemv_host(sets[r][m], N, K, xh[m], yh[m], xs[m], ys[m], stream=s_m, fmt=fmt)
+            join = torch.cuda.Event()
+            join.record(s_m)
+            stream.wait_event(join)
 
     # the host-buffer calls of a step are captured once per layer copy, like the device-resident steps
     e2e_graphs = None
@@ -455,6 +467,13 @@ def run_gpu(args):
     e2e_value = job_throughput_gbs(e2e_ms / e2e_steps, world)
     h2d = sum(2 * LLAMA3_8B[m][1] for m in MATRICES)
     d2h = sum(2 * LLAMA3_8B[m][0] for m in MATRICES)
+    # what the host-buffer calls left in pinned memory, against the same oracle rows
+    e2e_parity_ok = None
+    if rank == 0:
+        e2e_parity_ok = True
+        for m, (rows, ref, x) in refs.items():
+            rel, mab, bound = parity_metrics(yh[m].numpy()[rows], ref, x)[0]
+            e2e_parity_ok = bool(e2e_parity_ok and rel <= 1e-3 and mab <= bound)
 
     # ---- per-shape detail: steady state over rotating buffers > 2x L2, and isolated cold calls ----
     detail = {}
@@ -658,8 +677,9 @@ def run_gpu(args):
                      "kernel": "%s (7 launches per step; mean over the step)" % KERNEL_NAME[fmt],
                      "bytes_per_launch_mean": STEP_BYTES / 7.0, "us_per_launch_mean": 1e3 * ms_per_step / 7.0},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "us_per_layer": 1e3 * e2e_ms / e2e_steps,
-                "launch": ("cuda graph of the 7 ptqtp_gemv_host calls" if e2e_graphs else "plain calls")
+                "steps": e2e_steps, "us_per_layer": 1e3 * e2e_ms / e2e_steps, "parity_ok": e2e_parity_ok,
+                "launch": ("cuda graph of the 7 ptqtp_gemv_host calls, each on a stream of its own forked from the step's stream"
+                           if e2e_graphs else "plain calls, each on a stream of its own forked from the step's stream")
                           + ", one stream synchronisation per step"},
         "gpu_launches": launches, "clocks": clocks, "parity": parity, "shapes": detail,
     }
