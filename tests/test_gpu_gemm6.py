@@ -130,3 +130,35 @@ def test_bounded_wait_gives_up_reports_and_recovers(k_split):
         Y = _run(c, packed, N, K, k_split=k_split)
     assert_parity(Y, ref, c["x"], "after the failure")
     assert binding.ptqtp_kernel_status() == 0
+
+
+def test_many_launches_on_two_streams_give_the_same_bits():
+    # tensor memory is allocated and freed by every CTA: launches that share the SMs (two streams, back to back) must
+    # neither starve one another nor change a result
+    N, K = 2400, 2048
+    cs = [make_case(N, K, seed=300 + i, M=M) for i, M in enumerate((9, 24, 40, 64))]
+    packed = [pack_case(c, V3) for c in cs]
+    xs = [dev(c["x"]) for c in cs]
+    want = []
+    for c, p, x in zip(cs, packed, xs):
+        want.append(binding.ptqtp_gemm_skinny_cfg(p, N, K, x, path=6).cpu().numpy().view(np.uint16))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [[torch.empty((x.shape[0], N), dtype=torch.float16, device="cuda") for x in xs] for _ in range(2)]
+    torch.cuda.synchronize()
+    for rep in range(25):
+        for si, st in enumerate(streams):
+            with torch.cuda.stream(st):
+                for i in range(4):
+                    j = (i + si + rep) % 4
+                    binding.ptqtp_gemm_skinny_cfg(packed[j], N, K, xs[j], Y=outs[si][j], path=6, k_split=(1, 2, 4)[rep % 3],
+                                                  stream=st)
+    torch.cuda.synchronize()
+    assert binding.ptqtp_kernel_status() == 0
+    # the sum over a cluster is in rank order, but the split changes which partial sums exist: compare like with like
+    for si in range(2):
+        for j in range(4):
+            got = outs[si][j].cpu().numpy()
+            assert_parity(got, oracle_y(cs[j]), cs[j]["x"], "stream %d case %d" % (si, j))
+    for j in range(4):
+        a = binding.ptqtp_gemm_skinny_cfg(packed[j], N, K, xs[j], path=6).cpu().numpy().view(np.uint16)
+        assert np.array_equal(a, want[j])
