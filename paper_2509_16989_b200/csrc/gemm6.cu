@@ -2,20 +2,24 @@
 // fifth-generation tensor cores (tcgen05.mma, accumulators in tensor memory):
 //     Y[m] = alpha1 (.) (T1 X[m]) + alpha2 (.) (T2 X[m]),   m < M <= 64.
 //
-// A CTA of 128 threads owns 128 weight rows (8 tiles per superblock, contiguous in the blob); thread i is row i of
-// every MMA.  Per scale group of 128 columns:
-//   * each thread turns its row's 2-bit codes into fp16 trits (-1, 0, +1) with a byte-permute lookup -- the code in
-//     the high nibble of a selector byte picks the high byte of the fp16 value, the low nibble picks a zero byte --
-//     and writes them to tensor memory (tcgen05.st, one lane per row, 64 columns per plane): the A operand never
-//     passes through shared memory;
+// A CTA owns 128 weight rows (8 tiles per superblock, contiguous in the blob); row i is lane i of every MMA.  Ten
+// warps: eight decode (two threads per row, half of a group's columns each), one issues the MMAs, one copies the
+// code stages.  Per scale group of 128 columns:
+//   * the decoders turn their row's 2-bit codes into fp16 trits (-1, 0, +1): a mask per plane, two byte permutes that
+//     put two code bytes under the exponent of 1024, one fp16 FMA that maps 1024 + code * 2^s to code - 1; the trits
+//     go to tensor memory (tcgen05.st, one lane per row, 64 columns per plane): the A operand never passes through
+//     shared memory;
 //   * the activations of the group, fp16 as given (no quantisation), are the B operand: M rows padded to a multiple
 //     of 16, in shared memory as K-major core matrices (8 rows x 16 bytes), fetched with 16-byte cp.async one group
 //     ahead;
-//   * one thread issues 16 MMAs of 128 x NPAD x 16 (8 k-steps for each plane) into two fp32 accumulators and commits
-//     them to an mbarrier; the trits are exact in fp16, so each accumulator is the fp32 sum of +-x;
-//   * every thread reads its lane of both accumulators (tcgen05.ld) and adds alpha1 * d1 + alpha2 * d2 in fp32 to its
-//     NPAD running sums.
-// Two CTAs share an SM (256 of the 512 tensor-memory columns and about 100 KB of shared memory each), so one CTA's
+//   * an elected lane of the MMA warp issues 16 MMAs of 128 x NPAD x 16 (8 k-steps for each plane, in two halves of
+//     four k-steps that are decoded and multiplied alternately) into two fp32 accumulators and commits each half to
+//     an mbarrier; the trits are exact in fp16, so each accumulator is the fp32 sum of +-x;
+//   * the decoders read their lane of both accumulators (tcgen05.ld, half of the columns each) and add
+//     alpha1 * d1 + alpha2 * d2 in fp32 to their running sums.
+// The code stages are copied with 16-byte cp.async that regroup the lane entries of the tiles (made for warp-MMA
+// fragments) so that a warp of row threads reads 16 consecutive entries: no bank conflicts.
+// Two CTAs share an SM (256 of the 512 tensor-memory columns and 78 to 103 KB of shared memory each), so one CTA's
 // decode and epilogue run under the other's MMAs.  Matrices with few rows split K over a cluster of up to 8 CTAs;
 // the partial sums meet in distributed shared memory and are added in rank order (no atomics, reproducible).
 //
